@@ -1,0 +1,178 @@
+"""ctypes binding of the CPU oracle (oracle/cb_oracle.cpp).  TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the benchmark's cpu-baseline leg import this module; the CUDA path never
+does and shares nothing with it.  The shared object is compiled with g++ on first use.
+"""
+import ctypes as C
+import os
+import subprocess
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "cb_oracle.cpp")
+_SO = os.path.join(_HERE, "libcb_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        tmp = _SO + ".tmp%d" % os.getpid()
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-o", tmp, _SRC])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        L = _lib
+        L.orc_table_new.restype = C.c_void_p
+        L.orc_table_new.argtypes = [C.c_int] * 5
+        L.orc_table_free.argtypes = [C.c_void_p]
+        L.orc_table_reset.argtypes = [C.c_void_p]
+        L.orc_table_clock.restype = C.c_uint64
+        L.orc_table_clock.argtypes = [C.c_void_p]
+        L.orc_table_num_leaders.restype = C.c_int64
+        L.orc_table_num_leaders.argtypes = [C.c_void_p]
+        L.orc_insert.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.orc_query.restype = C.c_int
+        L.orc_query.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.orc_update.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int]
+        L.orc_table_dump.restype = C.c_int64
+        L.orc_table_dump.argtypes = [C.c_void_p] * 4
+        L.orc_draft_tree.restype = C.c_int
+        L.orc_draft_tree.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int] + [C.c_void_p] * 6
+        L.orc_tree_mask.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+        L.orc_argmax_f32.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_void_p]
+        L.orc_accept.restype = C.c_int
+        L.orc_accept.argtypes = [C.c_void_p] * 3 + [C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+        L.orc_tree_attn_rows.argtypes = ([C.c_void_p] * 8 + [C.c_int] * 6 + [C.c_double, C.c_void_p, C.c_int,
+                                                                               C.c_void_p, C.c_void_p])
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+class OracleTable:
+    """One sequence's cache table (Section 3.1)."""
+
+    def __init__(self, LL, FL, LC, FC, refresh_on_reinsert=True):
+        self.LL, self.FL, self.LC, self.FC = LL, FL, LC, FC
+        self._h = lib().orc_table_new(LL, FL, LC, FC, int(refresh_on_reinsert))
+
+    def __del__(self):
+        if getattr(self, "_h", None) and _lib is not None:
+            _lib.orc_table_free(self._h)
+            self._h = None
+
+    def reset(self):
+        lib().orc_table_reset(self._h)
+
+    @property
+    def clock(self):
+        return int(lib().orc_table_clock(self._h))
+
+    def __len__(self):
+        return int(lib().orc_table_num_leaders(self._h))
+
+    def insert(self, leader, follower):
+        L, F = _i32(leader), _i32(follower)
+        assert L.size == self.LL and F.size == self.FL
+        lib().orc_insert(self._h, _p(L), _p(F))
+
+    def query(self, leader):
+        L = _i32(leader)
+        assert L.size == self.LL
+        out = np.empty((self.FC, self.FL), dtype=np.int32)
+        n = lib().orc_query(self._h, _p(L), _p(out))
+        return [tuple(int(x) for x in out[i]) for i in range(n)]
+
+    def update(self, tokens, n_old, n_new):
+        s = _i32(tokens)
+        assert n_new <= s.size
+        lib().orc_update(self._h, _p(s), int(n_old), int(n_new))
+
+    def dump(self):
+        """[(leader tuple, [follower tuples])] — leaders and followers least recently used first."""
+        n = len(self)
+        leaders = np.empty((n, self.LL), dtype=np.int32)
+        nfol = np.empty(n, dtype=np.int32)
+        fol = np.empty((n, self.FC, self.FL), dtype=np.int32)
+        lib().orc_table_dump(self._h, _p(leaders), _p(nfol), _p(fol))
+        return [(tuple(int(x) for x in leaders[i]), [tuple(int(x) for x in fol[i, j]) for j in range(nfol[i])])
+                for i in range(n)]
+
+    def dump_arrays(self):
+        n = len(self)
+        leaders = np.empty((n, self.LL), dtype=np.int32)
+        nfol = np.empty(n, dtype=np.int32)
+        fol = np.empty((n, self.FC, self.FL), dtype=np.int32)
+        lib().orc_table_dump(self._h, _p(leaders), _p(nfol), _p(fol))
+        return leaders, nfol, fol
+
+    def draft_tree(self, tokens, seq_len, T, crt, max_depth, with_log=False):
+        s = _i32(tokens)
+        W = (T + 31) // 32
+        tok = np.empty(T, dtype=np.int32)
+        par = np.empty(T, dtype=np.int32)
+        dep = np.empty(T, dtype=np.int32)
+        mask = np.empty((T, W), dtype=np.uint32)
+        log = np.full((max(T, 1) * 2, self.LL + 1), -1, dtype=np.int32)
+        nq = C.c_int32(0)
+        n = lib().orc_draft_tree(self._h, _p(s), int(seq_len), T, crt, max_depth, _p(tok), _p(par), _p(dep),
+                                 _p(mask), _p(log), C.addressof(nq))
+        if with_log:
+            return n, tok, par, dep, mask, [(tuple(int(x) for x in r[:-1]), int(r[-1])) for r in log[: nq.value]]
+        return n, tok, par, dep, mask
+
+
+def tree_mask(par, n, T):
+    par = _i32(par)
+    mask = np.empty((T, (T + 31) // 32), dtype=np.uint32)
+    lib().orc_tree_mask(_p(par), int(n), int(T), _p(mask))
+    return mask
+
+
+def argmax_rows(logits):
+    x = np.ascontiguousarray(logits, dtype=np.float32)
+    assert x.ndim == 2
+    out = np.empty(x.shape[0], dtype=np.int32)
+    lib().orc_argmax_f32(_p(x), x.shape[0], x.shape[1], x.shape[1], _p(out))
+    return out
+
+
+def accept(tok, par, dep, n, target, dmax):
+    tok, par, dep, target = _i32(tok), _i32(par), _i32(dep), _i32(target)
+    nodes = np.empty(dmax, dtype=np.int32)
+    out = np.empty(dmax + 1, dtype=np.int32)
+    m = lib().orc_accept(_p(tok), _p(par), _p(dep), int(n), _p(target), int(dmax), _p(nodes), _p(out))
+    return m, nodes, out
+
+
+def tree_attn_rows(q, k_pool, v_pool, block_table, ctx_len, k_tree, v_tree, tree_mask_, rows, scale=None):
+    """All tensors in the library's layouts, bf16 as uint16 bit patterns. rows: int32 [n, 3] = (b, head, node).
+    Returns (out float64 [n, D], lse float64 [n])."""
+    q = np.ascontiguousarray(q, dtype=np.uint16)
+    k_pool = np.ascontiguousarray(k_pool, dtype=np.uint16)
+    v_pool = np.ascontiguousarray(v_pool, dtype=np.uint16)
+    k_tree = np.ascontiguousarray(k_tree, dtype=np.uint16)
+    v_tree = np.ascontiguousarray(v_tree, dtype=np.uint16)
+    bt, cl = _i32(block_table), _i32(ctx_len)
+    m = np.ascontiguousarray(tree_mask_, dtype=np.uint32)
+    rows = _i32(rows).reshape(-1, 3)
+    B, T, Hq, D = q.shape
+    _, P, Hkv, _ = k_pool.shape
+    assert k_tree.shape == (B, T, Hkv, D) and m.shape == (B, T, (T + 31) // 32)
+    out = np.empty((rows.shape[0], D), dtype=np.float64)
+    lse = np.empty(rows.shape[0], dtype=np.float64)
+    lib().orc_tree_attn_rows(_p(q), _p(k_pool), _p(v_pool), _p(bt), _p(cl), _p(k_tree), _p(v_tree), _p(m),
+                             T, Hq, Hkv, D, P, bt.shape[1], float(scale if scale is not None else D ** -0.5),
+                             _p(rows), rows.shape[0], _p(out), _p(lse))
+    return out, lse
