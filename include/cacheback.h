@@ -1,0 +1,228 @@
+/*
+ * cacheback.h — C ABI of the Cacheback draft-and-verify step on one NVIDIA B200 (sm_100a).
+ *
+ * One decoding step of Cacheback speculative decoding (paper Section 3) is, per sequence of a batch:
+ *   cb_update      slide a window over the newly accepted tokens and insert every leader->follower pair
+ *                  into the sequence's LRU cache table                       (Section 3.1; 3.2 last par.)
+ *   cb_draft_tree  grow a draft token tree by recursive table queries, breadth first, and emit parent
+ *                  indices, depths and the ancestor ("tree attention") mask  (Section 3.2)
+ *   cb_tree_attn   let every tree token attend to the sequence's paged KV cache plus its tree ancestors
+ *                  (the attention of the single verification forward pass)    (Section 3.2)
+ *   cb_accept      take the target's greedy choice after every node and keep the longest verified
+ *                  branch plus one more token                                 (Section 3.2)
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller unless a parameter says "host".
+ *     The library never allocates or frees device memory: all of its state and scratch lives in the
+ *     workspace handed to cb_create.
+ *   - `stream` is a cudaStream_t passed as void*. The four step calls and cb_reset only enqueue work
+ *     on it; they never synchronise.  Calls on one context must be ordered (same stream, or events).
+ *   - Host-detectable argument errors are returned at once and nothing is enqueued.  Conditions only
+ *     the device can see (a probe limit, a bounded wait that ran out) are recorded in a device status
+ *     word; the kernel finishes cleanly and cb_poll_status reports the first such code.
+ *   - Token ids are int32 >= 0; -1 is "no token".  Rows of per-node outputs beyond a sequence's node
+ *     count are padded: tokens / parents / depths / accepted nodes / emitted tokens with -1, mask and
+ *     attention rows with 0.
+ *   - bf16 tensors are passed as void* (16-bit brain floats, row-major, last index fastest).
+ */
+#ifndef CACHEBACK_H_
+#define CACHEBACK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cb_ctx cb_ctx; /* opaque */
+
+typedef enum {
+    CB_OK = 0,
+    CB_ERR_INVALID_ARG = 1,
+    CB_ERR_WORKSPACE_TOO_SMALL = 2,
+    CB_ERR_CUDA = 3,
+    CB_ERR_PROBE_LIMIT = 4, /* device: a hash probe visited every bucket without finding a free slot  */
+    CB_ERR_TIMEOUT = 5,     /* device: a bounded wait (mbarrier / flag) ran out                        */
+    CB_ERR_UNSUPPORTED = 6
+} cb_status;
+
+enum { CB_DTYPE_F32 = 0, CB_DTYPE_BF16 = 1 };
+
+/* cb_config.flags */
+enum {
+    CB_FLAG_NO_FOLLOWER_REFRESH = 1u, /* re-inserting a stored follower leaves its recency unchanged     */
+    CB_FLAG_ATTN_CUDA_CORES = 2u      /* run tree attention on the plain CUDA-core kernel (debug aid)    */
+};
+
+/*
+ * Shape of one context. Table parameters follow Section 3.1 / 3.2:
+ *   LL, FL  leader / follower length in tokens          (1..4, 1..8)
+ *   LC, FC  leader capacity per sequence, follower capacity per leader   (1..2^20, 1..16)
+ *   max_nodes  tree-size cap, root included: the paper's total draft length (TDL)   (1..128)
+ *   crt        nodes reserved for query levels >= 2: level 1 fills at most max(1, max_nodes - crt)
+ *   max_depth  deepest node depth allowed (root = 0)
+ * Attention shape: n_q_heads % n_kv_heads == 0, head_dim in {64, 128}, page_size == 16.
+ * vocab is the logits row length for cb_accept.
+ */
+typedef struct {
+    int32_t batch;
+    int32_t LL, FL, LC, FC;
+    int32_t max_nodes, crt, max_depth;
+    int32_t vocab;
+    int32_t n_q_heads, n_kv_heads, head_dim, page_size;
+    uint32_t flags;
+} cb_config;
+
+/* Bytes of device workspace cb_create needs for this shape (tables + scratch). Host call. */
+cb_status cb_workspace_bytes(const cb_config* cfg, size_t* bytes);
+
+/*
+ * Creates a context over caller-owned device memory `dev_workspace` (256-byte aligned, `bytes` long,
+ * on the current device) and empties every table.  Synchronises the device once.  *out is a small
+ * host object; the workspace must outlive it and belongs to the library until cb_destroy.
+ */
+cb_status cb_create(const cb_config* cfg, void* dev_workspace, size_t bytes, cb_ctx** out);
+
+/* Frees the host object only; never touches caller memory. NULL is allowed. */
+void cb_destroy(cb_ctx* ctx);
+
+/*
+ * Empties the tables of the sequences whose entry in dev_seq_mask ([batch] int32, non-zero = reset) is
+ * set, or of all sequences when dev_seq_mask is NULL (the per-task state reset of Section 4).
+ */
+cb_status cb_reset(cb_ctx* ctx, const int32_t* dev_seq_mask, void* stream);
+
+/*
+ * Table update (Section 3.1 insertion rules; Section 3.2 "sliding window over the accepted tokens";
+ * Section 3.3 prompt initialisation = the same call with n_old = 0).
+ *   tokens   int32 [batch, row_stride]  token history of every sequence
+ *   n_old    int32 [batch]  tokens already ingested by earlier calls
+ *   n_new    int32 [batch]  tokens valid now (n_new >= n_old; n_new <= row_stride)
+ * For sequence b every complete window i (leader = tokens[i .. i+LL), follower = tokens[i+LL ..
+ * i+LL+FL)) whose last token is new (i+LL+FL-1 in [n_old, n_new)) is inserted in increasing i:
+ * the leader is created (evicting the least recently used leader with its followers when LC are
+ * stored) or refreshed; the follower is appended (evicting the leader's least recently inserted
+ * follower when FC are stored) or, if already stored, refreshed.
+ */
+cb_status cb_update(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* n_old,
+                    const int32_t* n_new, void* stream);
+
+/*
+ * Draft-tree growth (Section 3.2).
+ *   tokens, row_stride  as in cb_update;  seq_len int32 [batch] = tokens valid per sequence
+ * Node 0 is the last token of the sequence (the one token whose K/V is not cached yet).  Level 1
+ * queries the table with the last LL tokens of the sequence; every later level queries, for each leaf
+ * that ends a complete follower, the last LL tokens of sequence ++ path-to-leaf.  Followers are
+ * attached most recently inserted first, each as a chain of FL nodes; growth is breadth first and stops
+ * at max_nodes (level 1 at max_nodes - crt), at max_depth, or when no leaf has a follower.  A chain
+ * that does not fit is cut short and not grown further.  Every issued query refreshes its leader.
+ * Outputs (all device):
+ *   tree_tokens, tree_parent, tree_depth  int32 [batch, max_nodes]   parent of node 0 is -1
+ *   tree_mask   uint32 [batch, max_nodes, W], W = ceil(max_nodes / 32): bit j of row i is set iff
+ *               node j is node i or an ancestor of it
+ *   n_nodes     int32 [batch]
+ * A sequence with seq_len < 1 gets n_nodes = 0; with fewer than LL tokens, the root only.
+ */
+cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* seq_len,
+                        int32_t* tree_tokens, int32_t* tree_parent, int32_t* tree_depth,
+                        uint32_t* tree_mask, int32_t* n_nodes, void* stream);
+
+/*
+ * Tree-masked attention over the paged KV cache (Section 3.2, "tree attention": a token attends only
+ * to its ancestors in the draft tree; the cached context is fully visible).
+ * With T = max_nodes, Hq / Hkv = n_q_heads / n_kv_heads, D = head_dim, P = page_size:
+ *   q            bf16 [batch, T, Hq, D]
+ *   k_pool,v_pool bf16 [num_pages, P, Hkv, D]   cached keys / values, paged
+ *   block_table  int32 [batch, max_pages]       page id of the j-th page of each sequence
+ *   ctx_len      int32 [batch]                  cached tokens per sequence (<= max_pages * P)
+ *   k_tree,v_tree bf16 [batch, T, Hkv, D]       keys / values of the tree tokens themselves
+ *   tree_mask    uint32 [batch, T, W], n_nodes int32 [batch]   as written by cb_draft_tree
+ *   out          bf16 [batch, T, Hq, D]         rows >= n_nodes are written as zero
+ *   lse          float [batch, Hq, T] or NULL   natural-log sum of exponentials per row (0 for padding)
+ *   max_ctx      host upper bound on every ctx_len (0 = max_pages * P); used only to size the grid
+ *   scale        softmax scale; 0 selects 1/sqrt(D)
+ * Row (b, i, h) = softmax_j(scale * q.k_j) v_j over j in {cached tokens of kv head h / (Hq/Hkv)}
+ * U {tree nodes in mask row i}; fp32 accumulation and softmax, output rounded to bf16.
+ * All base pointers must be 16-byte aligned.
+ */
+typedef struct {
+    const void* q;
+    const void* k_pool;
+    const void* v_pool;
+    const int32_t* block_table;
+    const int32_t* ctx_len;
+    const void* k_tree;
+    const void* v_tree;
+    const uint32_t* tree_mask;
+    const int32_t* n_nodes;
+    void* out;
+    float* lse;
+    int32_t max_pages;
+    int32_t num_pages;
+    int32_t max_ctx;
+    float scale;
+} cb_attn_args;
+
+cb_status cb_tree_attn(cb_ctx* ctx, const cb_attn_args* args, void* stream);
+
+/*
+ * Greedy acceptance (Section 3.2: the forward pass yields one more token than the accepted draft
+ * tokens, so a step emits between 1 and 1 + longest-branch tokens).
+ *   tree_tokens, tree_parent, tree_depth, n_nodes   as written by cb_draft_tree
+ *   logits        [batch, max_nodes, vocab] of logits_dtype (CB_DTYPE_F32 / CB_DTYPE_BF16), node rows
+ *                 logits_row_stride elements apart (sequence stride = max_nodes * logits_row_stride);
+ *                 finite values only.  target[i] = index of the first maximum of row i.
+ *   target_ids_in int32 [batch, max_nodes]: targets given directly.  Exactly one of logits /
+ *                 target_ids_in is non-NULL.
+ * Node i > 0 is verified iff its parent is verified and tree_tokens[i] == target[parent]; the root is
+ * verified.  The deepest verified node wins (lowest index among equally deep ones).  With m its depth:
+ *   n_accept       int32 [batch]               = m
+ *   accept_nodes   int32 [batch, max_depth]    the m nodes below the root on the winning path
+ *   out_tokens     int32 [batch, max_depth+1]  their tokens followed by target[winner]  (m+1 tokens)
+ *   target_ids_out int32 [batch, max_nodes] or NULL: the argmax of every valid row (-1 for padding)
+ */
+cb_status cb_accept(cb_ctx* ctx, const int32_t* tree_tokens, const int32_t* tree_parent,
+                    const int32_t* tree_depth, const int32_t* n_nodes, const void* logits,
+                    int32_t logits_dtype, int64_t logits_row_stride, const int32_t* target_ids_in,
+                    int32_t* n_accept, int32_t* accept_nodes, int32_t* out_tokens,
+                    int32_t* target_ids_out, void* stream);
+
+/*
+ * Canonical view of one sequence's table, for checkpointing and for comparing table contents:
+ * leaders least recently used first, each leader's followers least recently inserted first.
+ * HOST buffers: leaders int32 [LC, LL], n_followers int32 [LC], followers int32 [LC, FC, FL]
+ * (unused follower slots -1); any of them may be NULL.  *n_leaders receives the count.  Synchronises.
+ */
+cb_status cb_table_dump(cb_ctx* ctx, int32_t seq, int32_t* n_leaders, int32_t* leaders,
+                        int32_t* n_followers, int32_t* followers);
+
+/* Replaces one sequence's table by the given canonical content (same HOST layouts as cb_table_dump;
+ * recency = position). Synchronises. */
+cb_status cb_table_load(cb_ctx* ctx, int32_t seq, int32_t n_leaders, const int32_t* leaders,
+                        const int32_t* n_followers, const int32_t* followers);
+
+/*
+ * Reads (and clears) the device status word and copies the counters to the HOST array `counters`
+ * (CB_NUM_COUNTERS entries, may be NULL).  Synchronises.
+ */
+enum {
+    CB_CNT_INSERTS = 0,
+    CB_CNT_LEADER_EVICTIONS = 1,
+    CB_CNT_FOLLOWER_EVICTIONS = 2,
+    CB_CNT_QUERIES = 3,
+    CB_CNT_QUERY_HITS = 4,
+    CB_CNT_MAX_PROBE = 5,
+    CB_NUM_COUNTERS = 8
+};
+cb_status cb_poll_status(cb_ctx* ctx, cb_status* device_status, uint64_t* counters);
+
+/* Kernels launched by this library since the process started (host-side count). */
+uint64_t cb_launch_count(void);
+
+const char* cb_status_str(cb_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CACHEBACK_H_ */

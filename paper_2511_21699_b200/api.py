@@ -1,0 +1,182 @@
+"""Thin Python binding of the C-ABI library: argument marshalling only.
+
+Tensors are torch CUDA tensors (device memory and streams are torch's); every step of the path runs in
+the library's kernels.  Method names mirror the C entry points.
+"""
+import ctypes as C
+
+import numpy as np
+import torch
+
+from . import _lib
+from ._lib import CbConfigC, CbAttnArgsC
+
+
+class CachebackError(RuntimeError):
+    pass
+
+
+def _check(code, what):
+    if code != _lib.CB_OK:
+        raise CachebackError("%s failed: %s" % (what, _lib.load().cb_status_str(code).decode()))
+
+
+def _ptr(t, dtype=None):
+    if t is None:
+        return None
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous()):
+        raise CachebackError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise CachebackError("expected dtype %s, got %s" % (dtype, t.dtype))
+    return t.data_ptr()
+
+
+def _stream(stream):
+    return (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
+
+
+class Cacheback:
+    """One context: per-sequence tables plus scratch, in a workspace tensor owned by this object."""
+
+    def __init__(self, batch, LL, FL, LC, FC, max_nodes, crt, max_depth, vocab, n_q_heads, n_kv_heads, head_dim,
+                 page_size=16, flags=0, device="cuda:0"):
+        self.lib = _lib.load()
+        if not torch.cuda.is_available():
+            raise CachebackError("no CUDA device: the library has no CPU path")
+        self.device = torch.device(device)
+        self.cfg = CbConfigC(batch, LL, FL, LC, FC, max_nodes, crt, max_depth, vocab, n_q_heads, n_kv_heads, head_dim,
+                             page_size, flags)
+        nbytes = C.c_size_t(0)
+        _check(self.lib.cb_workspace_bytes(C.byref(self.cfg), C.byref(nbytes)), "cb_workspace_bytes")
+        self.workspace_bytes = nbytes.value
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
+            base = (self.workspace.data_ptr() + 255) // 256 * 256
+            h = C.c_void_p(None)
+            _check(self.lib.cb_create(C.byref(self.cfg), base, nbytes.value, C.byref(h)), "cb_create")
+        self._h = h
+        self.W = (max_nodes + 31) // 32
+
+    @classmethod
+    def from_config(cls, cfg, flags=0, device="cuda:0", batch=None):
+        """cfg: a workloads.CbConfig-like object."""
+        return cls(batch or cfg.batch, cfg.LL, cfg.FL, cfg.LC, cfg.FC, cfg.max_nodes, cfg.crt, cfg.max_depth, cfg.vocab,
+                   cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.page_size, flags, device)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self.lib.cb_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- the four step calls -----------------------------------------------------------------------
+    def cb_reset(self, seq_mask=None, stream=None):
+        _check(self.lib.cb_reset(self._h, _ptr(seq_mask, torch.int32), _stream(stream)), "cb_reset")
+
+    def cb_update(self, tokens, n_old, n_new, stream=None):
+        _check(self.lib.cb_update(self._h, _ptr(tokens, torch.int32), tokens.stride(0), _ptr(n_old, torch.int32),
+                                  _ptr(n_new, torch.int32), _stream(stream)), "cb_update")
+
+    def alloc_tree(self):
+        B, T = self.cfg.batch, self.cfg.max_nodes
+        i32 = dict(dtype=torch.int32, device=self.device)
+        return dict(tokens=torch.empty(B, T, **i32), parent=torch.empty(B, T, **i32), depth=torch.empty(B, T, **i32),
+                    mask=torch.empty(B, T, self.W, **i32), n_nodes=torch.empty(B, **i32))
+
+    def cb_draft_tree(self, tokens, seq_len, tree=None, stream=None):
+        tree = tree if tree is not None else self.alloc_tree()
+        _check(self.lib.cb_draft_tree(self._h, _ptr(tokens, torch.int32), tokens.stride(0), _ptr(seq_len, torch.int32),
+                                      _ptr(tree["tokens"], torch.int32), _ptr(tree["parent"], torch.int32),
+                                      _ptr(tree["depth"], torch.int32), _ptr(tree["mask"], torch.int32),
+                                      _ptr(tree["n_nodes"], torch.int32), _stream(stream)), "cb_draft_tree")
+        return tree
+
+    def cb_tree_attn(self, q, k_pool, v_pool, block_table, ctx_len, k_tree, v_tree, tree_mask, n_nodes, out=None,
+                     lse=None, max_ctx=0, scale=0.0, stream=None):
+        if out is None:
+            out = torch.empty_like(q)
+        a = CbAttnArgsC(_ptr(q, torch.bfloat16), _ptr(k_pool, torch.bfloat16), _ptr(v_pool, torch.bfloat16),
+                        _ptr(block_table, torch.int32), _ptr(ctx_len, torch.int32), _ptr(k_tree, torch.bfloat16),
+                        _ptr(v_tree, torch.bfloat16), _ptr(tree_mask, torch.int32), _ptr(n_nodes, torch.int32),
+                        _ptr(out, torch.bfloat16), _ptr(lse, torch.float32), block_table.shape[1], k_pool.shape[0],
+                        int(max_ctx), float(scale))
+        _check(self.lib.cb_tree_attn(self._h, C.byref(a), _stream(stream)), "cb_tree_attn")
+        return out
+
+    def alloc_accept(self):
+        B, Dm = self.cfg.batch, self.cfg.max_depth
+        i32 = dict(dtype=torch.int32, device=self.device)
+        return dict(n_accept=torch.empty(B, **i32), accept_nodes=torch.empty(B, Dm, **i32),
+                    out_tokens=torch.empty(B, Dm + 1, **i32), target_ids=torch.empty(B, self.cfg.max_nodes, **i32))
+
+    def cb_accept(self, tree, logits=None, target_ids=None, res=None, stream=None):
+        res = res if res is not None else self.alloc_accept()
+        dtype, stride, lp = 0, 0, None
+        if logits is not None:
+            if logits.dtype == torch.float32:
+                dtype = _lib.CB_DTYPE_F32
+            elif logits.dtype == torch.bfloat16:
+                dtype = _lib.CB_DTYPE_BF16
+            else:
+                raise CachebackError("logits must be float32 or bfloat16")
+            if not (logits.is_cuda and logits.dim() == 3 and logits.stride(2) == 1 and
+                    logits.stride(0) == logits.shape[1] * logits.stride(1)):
+                raise CachebackError("logits must be [batch, max_nodes, vocab] with a uniform row stride")
+            stride, lp = logits.stride(1), logits.data_ptr()
+        _check(self.lib.cb_accept(self._h, _ptr(tree["tokens"], torch.int32), _ptr(tree["parent"], torch.int32),
+                                  _ptr(tree["depth"], torch.int32), _ptr(tree["n_nodes"], torch.int32), lp, dtype, stride,
+                                  _ptr(target_ids, torch.int32), _ptr(res["n_accept"], torch.int32),
+                                  _ptr(res["accept_nodes"], torch.int32), _ptr(res["out_tokens"], torch.int32),
+                                  _ptr(res["target_ids"], torch.int32), _stream(stream)), "cb_accept")
+        return res
+
+    # ---- helpers ------------------------------------------------------------------------------------
+    def cb_table_dump(self, seq):
+        """[(leader tuple, [follower tuples])], least recently used first (host lists)."""
+        c = self.cfg
+        n = C.c_int32(0)
+        leaders = np.empty((c.LC, c.LL), dtype=np.int32)
+        nfol = np.empty(c.LC, dtype=np.int32)
+        fol = np.empty((c.LC, c.FC, c.FL), dtype=np.int32)
+        _check(self.lib.cb_table_dump(self._h, seq, C.byref(n), leaders.ctypes.data, nfol.ctypes.data, fol.ctypes.data),
+               "cb_table_dump")
+        return [(tuple(int(x) for x in leaders[i]), [tuple(int(x) for x in fol[i, j]) for j in range(nfol[i])])
+                for i in range(n.value)]
+
+    def cb_table_dump_arrays(self, seq):
+        c = self.cfg
+        n = C.c_int32(0)
+        leaders = np.empty((c.LC, c.LL), dtype=np.int32)
+        nfol = np.empty(c.LC, dtype=np.int32)
+        fol = np.empty((c.LC, c.FC, c.FL), dtype=np.int32)
+        _check(self.lib.cb_table_dump(self._h, seq, C.byref(n), leaders.ctypes.data, nfol.ctypes.data, fol.ctypes.data),
+               "cb_table_dump")
+        return leaders[: n.value], nfol[: n.value], fol[: n.value]
+
+    def cb_table_load(self, seq, table):
+        c = self.cfg
+        n = len(table)
+        leaders = np.zeros((max(n, 1), c.LL), dtype=np.int32)
+        nfol = np.zeros(max(n, 1), dtype=np.int32)
+        fol = np.full((max(n, 1), c.FC, c.FL), -1, dtype=np.int32)
+        for i, (L, fs) in enumerate(table):
+            leaders[i] = L
+            nfol[i] = len(fs)
+            for j, f in enumerate(fs):
+                fol[i, j] = f
+        _check(self.lib.cb_table_load(self._h, seq, n, leaders.ctypes.data, nfol.ctypes.data, fol.ctypes.data),
+               "cb_table_load")
+
+    def cb_poll_status(self):
+        st = C.c_int32(0)
+        cnt = np.zeros(_lib.CB_NUM_COUNTERS, dtype=np.uint64)
+        _check(self.lib.cb_poll_status(self._h, C.byref(st), cnt.ctypes.data), "cb_poll_status")
+        return st.value, dict(zip(_lib.COUNTER_NAMES, (int(x) for x in cnt)))
+
+    def launch_count(self):
+        return int(self.lib.cb_launch_count())

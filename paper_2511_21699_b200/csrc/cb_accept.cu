@@ -1,0 +1,240 @@
+// Greedy acceptance: streaming arg-max over the logits of every valid tree node, then a warp-level walk
+// that finds the longest verified path.  One launch: CTAs reduce chunks of logit rows into packed
+// (value, index) maxima with 64-bit atomic max; the last CTA of a sequence to finish walks its tree.
+#include "cb_common.cuh"
+
+namespace {
+
+// Order-preserving map of a finite float to uint32 (larger float -> larger integer). -0 is folded into +0
+// first so that equal values compare equal.
+__device__ __forceinline__ uint32_t f2ord(float x) {
+    x += 0.0f;
+    const uint32_t u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+// Packed key: larger value wins, then the smaller index.
+__device__ __forceinline__ unsigned long long pack(float x, uint32_t idx) {
+    return ((unsigned long long)f2ord(x) << 32) | (unsigned long long)(0xFFFFFFFFu - idx);
+}
+__device__ __forceinline__ unsigned long long umax64(unsigned long long a, unsigned long long b) { return a > b ? a : b; }
+
+__device__ __forceinline__ float4 ldg_stream4(const float* p) {
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint4 ldg_stream4u(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// Walk of one sequence by one warp (n <= 128 nodes, parents precede children).
+__device__ void accept_walk(int b, int T, int Dmax, const int32_t* __restrict__ tok, const int32_t* __restrict__ par,
+                            const int32_t* __restrict__ dep, int n, const int32_t* target_s /*shared, [T]*/,
+                            int32_t* __restrict__ n_accept, int32_t* __restrict__ accept_nodes,
+                            int32_t* __restrict__ out_tokens, int lane) {
+    const int32_t* tk = tok + (size_t)b * T;
+    const int32_t* pa = par + (size_t)b * T;
+    const int32_t* de = dep + (size_t)b * T;
+    // key = (depth << 8) | (255 - index) for verified nodes: max = deepest, lowest index among ties
+    uint32_t best = 0;
+    for (int i = lane; i < n; i += 32) {
+        bool good = true;
+        int c = i;
+        for (int guard = 0; guard < CB_MAX_T && c > 0; ++guard) {
+            const int p = pa[c];
+            if (p < 0 || p >= c) { good = false; break; }      // malformed tree: treat as unverified
+            good = good && (tk[c] == target_s[p]);
+            c = p;
+        }
+        if (good) best = max(best, ((uint32_t)de[i] << 8) | (uint32_t)(255 - i));
+    }
+    best = __reduce_max_sync(CB_FULL, best);
+    int node = n > 0 ? 255 - (int)(best & 255u) : 0;
+    int m = n > 0 ? (int)(best >> 8) : 0;
+    if (m > Dmax) m = Dmax;
+    for (int k = lane; k < Dmax; k += 32) accept_nodes[(size_t)b * Dmax + k] = -1;
+    for (int k = lane; k <= Dmax; k += 32) out_tokens[(size_t)b * (Dmax + 1) + k] = -1;
+    __syncwarp();
+    if (lane == 0) {
+        n_accept[b] = m;
+        if (n > 0) {
+            out_tokens[(size_t)b * (Dmax + 1) + m] = target_s[node];
+            int c = node;
+            for (int k = m - 1; k >= 0 && c > 0; --k) {
+                accept_nodes[(size_t)b * Dmax + k] = c;
+                out_tokens[(size_t)b * (Dmax + 1) + k] = tk[c];
+                c = pa[c];
+            }
+        }
+    }
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(256) cb_accept_logits_kernel(
+    int T, int V, int Dmax, int chunk, int chunks_per_row, const void* __restrict__ logits, int64_t row_stride,
+    const int32_t* __restrict__ tok, const int32_t* __restrict__ par, const int32_t* __restrict__ dep,
+    const int32_t* __restrict__ n_nodes, unsigned long long* rowmax, uint32_t* ticket,
+    int32_t* __restrict__ n_accept, int32_t* __restrict__ accept_nodes, int32_t* __restrict__ out_tokens,
+    int32_t* __restrict__ target_out) {
+    const int b = blockIdx.z, i = blockIdx.y, ck = blockIdx.x, tid = threadIdx.x;
+    const int n = n_nodes[b];
+    __shared__ unsigned long long s_red[8];
+    __shared__ int32_t s_target[CB_MAX_T];
+    __shared__ int s_last;
+    if (i < n) {
+        const int v0 = ck * chunk, v1 = min(V, v0 + chunk);
+        unsigned long long best = 0ull;
+        if (!BF16) {
+            const float* rowp = (const float*)logits + ((size_t)b * T + i) * row_stride;
+            // head up to a 16-byte boundary, vector body, scalar tail
+            int v = v0;
+            const uintptr_t a = (uintptr_t)(rowp + v);
+            int head = (int)(((16 - (a & 15)) & 15) >> 2);
+            head = min(head, v1 - v);
+            if (tid < head) best = pack(rowp[v + tid], (uint32_t)(v + tid));
+            v += head;
+            const int nvec = (v1 - v) >> 2;
+            const float* base = rowp + v;
+            for (int k = tid; k < nvec; k += blockDim.x * 4) {
+                float4 x[4];
+                int kk[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) { kk[u] = k + u * blockDim.x; if (kk[u] < nvec) x[u] = ldg_stream4(base + 4 * (size_t)kk[u]); }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) if (kk[u] < nvec) {
+                    const uint32_t id = (uint32_t)(v + 4 * kk[u]);
+                    best = umax64(best, pack(x[u].x, id));
+                    best = umax64(best, pack(x[u].y, id + 1));
+                    best = umax64(best, pack(x[u].z, id + 2));
+                    best = umax64(best, pack(x[u].w, id + 3));
+                }
+            }
+            const int tail0 = v + 4 * nvec;
+            if (tail0 + tid < v1) best = umax64(best, pack(rowp[tail0 + tid], (uint32_t)(tail0 + tid)));
+        } else {
+            const __nv_bfloat16* rowp = (const __nv_bfloat16*)logits + ((size_t)b * T + i) * row_stride;
+            int v = v0;
+            const uintptr_t a = (uintptr_t)(rowp + v);
+            int head = (int)(((16 - (a & 15)) & 15) >> 1);
+            head = min(head, v1 - v);
+            if (tid < head) best = pack(__bfloat162float(rowp[v + tid]), (uint32_t)(v + tid));
+            v += head;
+            const int nvec = (v1 - v) >> 3;
+            const __nv_bfloat16* base = rowp + v;
+            for (int k = tid; k < nvec; k += blockDim.x * 4) {
+                uint4 x[4];
+                int kk[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) { kk[u] = k + u * blockDim.x; if (kk[u] < nvec) x[u] = ldg_stream4u(base + 8 * (size_t)kk[u]); }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) if (kk[u] < nvec) {
+                    const uint32_t id = (uint32_t)(v + 8 * kk[u]);
+                    const uint32_t wds[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        best = umax64(best, pack(__uint_as_float(wds[q] << 16), id + 2 * q));
+                        best = umax64(best, pack(__uint_as_float(wds[q] & 0xFFFF0000u), id + 2 * q + 1));
+                    }
+                }
+            }
+            const int tail0 = v + 8 * nvec;
+            if (tail0 + tid < v1) best = umax64(best, pack(__bfloat162float(rowp[tail0 + tid]), (uint32_t)(tail0 + tid)));
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) best = umax64(best, __shfl_xor_sync(CB_FULL, best, o));
+        if ((tid & 31) == 0) s_red[tid >> 5] = best;
+        __syncthreads();
+        if (tid == 0) {
+            for (int w = 1; w < (int)(blockDim.x >> 5); ++w) best = umax64(best, s_red[w]);
+            atomicMax(&rowmax[(size_t)b * T + i], best);
+        }
+    }
+    // The last CTA of this sequence to arrive owns the walk (and re-zeroes the scratch for the next call).
+    if (tid == 0) {
+        __threadfence();
+        const uint32_t total = gridDim.x * gridDim.y;
+        s_last = (atomicAdd(&ticket[b], 1u) == total - 1u) ? 1 : 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int k = tid; k < T; k += blockDim.x) {
+        int32_t tg = -1;
+        if (k < n) {
+            const unsigned long long r = atomicExch(&rowmax[(size_t)b * T + k], 0ull);
+            tg = (int32_t)(0xFFFFFFFFu - (uint32_t)(r & 0xFFFFFFFFull));
+        }
+        s_target[k] = tg;
+        if (target_out) target_out[(size_t)b * T + k] = tg;
+    }
+    if (tid == 0) ticket[b] = 0u;
+    __syncthreads();
+    if (tid < 32) accept_walk(b, T, Dmax, tok, par, dep, n, s_target, n_accept, accept_nodes, out_tokens, tid);
+}
+
+__global__ void __launch_bounds__(128) cb_accept_ids_kernel(int B, int T, int Dmax, const int32_t* __restrict__ target_in,
+                                                            const int32_t* __restrict__ tok, const int32_t* __restrict__ par,
+                                                            const int32_t* __restrict__ dep, const int32_t* __restrict__ n_nodes,
+                                                            int32_t* __restrict__ n_accept, int32_t* __restrict__ accept_nodes,
+                                                            int32_t* __restrict__ out_tokens, int32_t* __restrict__ target_out) {
+    __shared__ int32_t s_target[4][CB_MAX_T];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int b = blockIdx.x * 4 + w;
+    if (b >= B) return;
+    const int n = n_nodes[b];
+    for (int k = lane; k < T; k += 32) {
+        const int32_t tg = k < n ? target_in[(size_t)b * T + k] : -1;
+        s_target[w][k] = tg;
+        if (target_out) target_out[(size_t)b * T + k] = tg;
+    }
+    __syncwarp();
+    accept_walk(b, T, Dmax, tok, par, dep, n, s_target[w], n_accept, accept_nodes, out_tokens, lane);
+}
+
+}  // namespace
+
+extern "C" cb_status cb_accept(cb_ctx* ctx, const int32_t* tree_tokens, const int32_t* tree_parent,
+                               const int32_t* tree_depth, const int32_t* n_nodes, const void* logits,
+                               int32_t logits_dtype, int64_t logits_row_stride, const int32_t* target_ids_in,
+                               int32_t* n_accept, int32_t* accept_nodes, int32_t* out_tokens,
+                               int32_t* target_ids_out, void* stream) {
+    CB_CHECK_ARG(ctx && tree_tokens && tree_parent && tree_depth && n_nodes && n_accept && accept_nodes && out_tokens);
+    CB_CHECK_ARG((logits != nullptr) != (target_ids_in != nullptr));
+    const cb_config& c = ctx->cfg;
+    const int T = c.max_nodes, Dmax = c.max_depth;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (target_ids_in) {
+        cb_accept_ids_kernel<<<(c.batch + 3) / 4, 128, 0, st>>>(c.batch, T, Dmax, target_ids_in, tree_tokens, tree_parent,
+                                                                 tree_depth, n_nodes, n_accept, accept_nodes, out_tokens,
+                                                                 target_ids_out);
+    } else {
+        CB_CHECK_ARG(logits_dtype == CB_DTYPE_F32 || logits_dtype == CB_DTYPE_BF16);
+        CB_CHECK_ARG(logits_row_stride >= c.vocab);
+        const int esz = logits_dtype == CB_DTYPE_F32 ? 4 : 2;
+        CB_CHECK_ARG(((uintptr_t)logits & (esz - 1)) == 0);
+        // chunk: about 32 KB of a row per CTA, fewer chunks when the batch alone fills the machine
+        int chunk = 32768 / esz;
+        const long rows = (long)c.batch * T;
+        if (rows >= 8L * ctx->num_sms) chunk *= 4;
+        int cpr = (c.vocab + chunk - 1) / chunk;
+        chunk = ((c.vocab + cpr - 1) / cpr + 7) & ~7;
+        cpr = (c.vocab + chunk - 1) / chunk;
+        dim3 grid(cpr, T, c.batch);
+        if (c.batch > 65535) return CB_ERR_UNSUPPORTED;
+        if (logits_dtype == CB_DTYPE_F32)
+            cb_accept_logits_kernel<false><<<grid, 256, 0, st>>>(T, c.vocab, Dmax, chunk, cpr, logits, logits_row_stride,
+                                                                 tree_tokens, tree_parent, tree_depth, n_nodes, ctx->d_rowmax,
+                                                                 ctx->d_ticket, n_accept, accept_nodes, out_tokens, target_ids_out);
+        else
+            cb_accept_logits_kernel<true><<<grid, 256, 0, st>>>(T, c.vocab, Dmax, chunk, cpr, logits, logits_row_stride,
+                                                                tree_tokens, tree_parent, tree_depth, n_nodes, ctx->d_rowmax,
+                                                                ctx->d_ticket, n_accept, accept_nodes, out_tokens, target_ids_out);
+    }
+    cb_count_launch(1);
+    CB_CUDA(cudaGetLastError());
+    return CB_OK;
+}

@@ -1,0 +1,98 @@
+// Shared declarations of the library: context object, workspace layout, table view, hashing.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "cacheback.h"
+
+#define CB_FULL 0xFFFFFFFFu
+#define CB_IDX_EMPTY 0u
+#define CB_IDX_TOMB 0xFFFFFFFFu
+#define CB_EID_BITS 20
+#define CB_EID_MASK ((1u << CB_EID_BITS) - 1u)
+#define CB_MAX_T 128
+#define CB_MAX_LL 4
+#define CB_MAX_FL 8
+#define CB_MAX_FC 16
+
+// Per-sequence table in the workspace (all 32-bit words):
+//   hdr[4]            clock, leader count, unused, unused
+//   index[nslots]     open-addressing index over 32-slot buckets: 0 = empty, 0xFFFFFFFF = deleted,
+//                     else (tag << 20) | entry id, tag in [1, 4094] taken from the key's hash
+//   lstamp[LC]        leader recency stamps (dense, so the LRU scan reads 4 bytes per leader)
+//   entries[LC][E]    key[LL], follower stamps[FC] (0 = free), follower tokens[FC][FL]; E padded to 4 words
+struct CbTables {
+    uint32_t* hdr;
+    uint32_t* index;
+    uint32_t* lstamp;
+    uint32_t* entries;
+    uint32_t nslots, E;
+    int32_t LL, FL, LC, FC;
+    uint32_t refresh;  // re-inserting a stored follower refreshes it
+};
+
+struct CbSeq {  // one sequence's slice of CbTables
+    uint32_t* hdr;
+    uint32_t* index;
+    uint32_t* lstamp;
+    uint32_t* entries;
+};
+
+__device__ __forceinline__ CbSeq cb_seq(const CbTables& t, int b) {
+    CbSeq s;
+    s.hdr = t.hdr + (size_t)b * 4;
+    s.index = t.index + (size_t)b * t.nslots;
+    s.lstamp = t.lstamp + (size_t)b * t.LC;
+    s.entries = t.entries + (size_t)b * t.LC * t.E;
+    return s;
+}
+
+__host__ __device__ __forceinline__ uint64_t cb_hash4(int32_t k0, int32_t k1, int32_t k2, int32_t k3, int LL) {
+    uint64_t h = 0x9E3779B97F4A7C15ull ^ (uint64_t)LL;
+    h = (h ^ (uint32_t)k0) * 0xFF51AFD7ED558CCDull; h ^= h >> 32;
+    if (LL > 1) { h = (h ^ (uint32_t)k1) * 0xFF51AFD7ED558CCDull; h ^= h >> 32; }
+    if (LL > 2) { h = (h ^ (uint32_t)k2) * 0xFF51AFD7ED558CCDull; h ^= h >> 32; }
+    if (LL > 3) { h = (h ^ (uint32_t)k3) * 0xFF51AFD7ED558CCDull; h ^= h >> 32; }
+    h ^= h >> 33; h *= 0xC4CEB9FE1A85EC53ull; h ^= h >> 33;
+    return h;
+}
+__host__ __device__ __forceinline__ uint32_t cb_hash_tag(uint64_t h) { return (uint32_t)(h & 0xFFFFFFFFull) % 4094u + 1u; }
+__host__ __device__ __forceinline__ uint32_t cb_hash_bucket(uint64_t h, uint32_t nslots) {
+    return (uint32_t)(h >> 32) & ((nslots >> 5) - 1u);
+}
+
+struct cb_ctx {
+    cb_config cfg;
+    int device;
+    char* ws;
+    size_t ws_bytes;
+    CbTables tables;
+    uint32_t* d_status;     // [4]
+    unsigned long long* d_counters;  // [CB_NUM_COUNTERS]
+    unsigned long long* d_rowmax;    // [batch * max_nodes] packed (value, index) maxima, zero between calls
+    uint32_t* d_ticket;     // [batch] CTAs-finished counters, zero between calls
+    float* d_attn_part;     // split-KV partial outputs
+    size_t attn_part_floats;
+    int attn_max_units;     // partial slots available
+    int num_sms;
+};
+
+struct CbLayout {
+    uint32_t nslots, E;
+    size_t off_hdr, off_index, off_lstamp, off_entries, off_status, off_counters, off_rowmax, off_ticket,
+        off_attn_part, attn_part_floats, total;
+    int attn_max_units;
+};
+
+cb_status cb_compute_layout(const cb_config* cfg, CbLayout* L);
+void cb_count_launch(int n);
+
+#define CB_ATTN_MAX_UNITS 1024  // split-KV partial slots (each 128 rows x (D + 4) floats)
+
+#define CB_CHECK_ARG(cond) do { if (!(cond)) return CB_ERR_INVALID_ARG; } while (0)
+#include <stdio.h>
+// CUDA failures are exceptional: say where and what on stderr, then report CB_ERR_CUDA.
+#define CB_CUDA(call) do { cudaError_t cb_e_ = (call); if (cb_e_ != cudaSuccess) { \
+    fprintf(stderr, "cacheback: %s:%d: %s\n", __FILE__, __LINE__, cudaGetErrorString(cb_e_)); return CB_ERR_CUDA; } } while (0)

@@ -1,0 +1,352 @@
+// Per-sequence LRU cache table kernels: sliding-window update and batched draft-tree expansion.
+//
+// Every table operation is executed by one warp acting as a unit: the 32 lanes probe the 32 slots of an
+// index bucket with one coalesced load, compare the FC followers of an entry in parallel, and scan the
+// dense stamp array for the least recently used leader.  Recency is a per-sequence operation counter
+// ("clock"); a leader or follower stamp is the clock value of the operation that last touched it.
+#include "cb_common.cuh"
+
+namespace {
+
+struct Probe {
+    int eid;             // entry id, -1 absent, -2 probe limit
+    uint32_t slot;       // index slot holding the entry (when found)
+    uint32_t free_slot;  // first reusable slot on the probe path (when absent), 0xFFFFFFFF if none seen
+    uint32_t probes;     // buckets visited
+};
+
+// Warp-wide lookup of a leader. mykey = key[lane] for lane < LL (0 otherwise), identical call in all lanes.
+__device__ __forceinline__ Probe tbl_find(const CbTables& t, const CbSeq& s, int32_t mykey, uint64_t h, int lane) {
+    Probe r;
+    r.eid = -2; r.slot = 0; r.free_slot = 0xFFFFFFFFu; r.probes = 0;
+    const uint32_t nb = t.nslots >> 5, tag = cb_hash_tag(h);
+    uint32_t bucket = cb_hash_bucket(h, t.nslots);
+    for (uint32_t p = 0; p < nb; ++p) {
+        r.probes = p + 1;
+        const uint32_t w = s.index[bucket * 32 + lane];
+        uint32_t cand = __ballot_sync(CB_FULL, w != CB_IDX_EMPTY && w != CB_IDX_TOMB && (w >> CB_EID_BITS) == tag);
+        while (cand) {
+            const int l = __ffs(cand) - 1;
+            cand &= cand - 1;
+            const uint32_t eid = __shfl_sync(CB_FULL, w, l) & CB_EID_MASK;
+            bool eq = true;
+            if (lane < t.LL) eq = ((int32_t)s.entries[(size_t)eid * t.E + lane] == mykey);
+            if (__all_sync(CB_FULL, eq)) { r.eid = (int)eid; r.slot = bucket * 32 + l; return r; }
+        }
+        const uint32_t fr = __ballot_sync(CB_FULL, w == CB_IDX_EMPTY || w == CB_IDX_TOMB);
+        if (r.free_slot == 0xFFFFFFFFu && fr) r.free_slot = bucket * 32 + (__ffs(fr) - 1);
+        if (__ballot_sync(CB_FULL, w == CB_IDX_EMPTY)) { r.eid = -1; return r; }
+        bucket = (bucket + 1) & (nb - 1);
+    }
+    return r;
+}
+
+__device__ __forceinline__ uint64_t warp_hash(const CbTables& t, int32_t mykey) {
+    const int32_t k0 = __shfl_sync(CB_FULL, mykey, 0), k1 = __shfl_sync(CB_FULL, mykey, 1),
+                  k2 = __shfl_sync(CB_FULL, mykey, 2), k3 = __shfl_sync(CB_FULL, mykey, 3);
+    return cb_hash4(k0, k1, k2, k3, t.LL);
+}
+
+// Removes the least recently used leader from the index and returns its entry id for reuse.
+__device__ int tbl_evict_lru(const CbTables& t, const CbSeq& s, int lane, uint32_t* status) {
+    uint32_t minv = 0xFFFFFFFFu;
+    int mine = 0;
+#pragma unroll 4
+    for (int i = lane; i < t.LC; i += 32) {
+        const uint32_t v = s.lstamp[i];
+        if (v < minv) { minv = v; mine = i; }
+    }
+    const uint32_t g = __reduce_min_sync(CB_FULL, minv);
+    const int wl = __ffs(__ballot_sync(CB_FULL, minv == g)) - 1;   // stamps are unique
+    const int eid = __shfl_sync(CB_FULL, mine, wl);
+    const int32_t vkey = lane < t.LL ? (int32_t)s.entries[(size_t)eid * t.E + lane] : 0;
+    const uint64_t h = warp_hash(t, vkey);
+    const uint32_t nb = t.nslots >> 5, word = (cb_hash_tag(h) << CB_EID_BITS) | (uint32_t)eid;
+    uint32_t bucket = cb_hash_bucket(h, t.nslots);
+    for (uint32_t p = 0; p < nb; ++p) {
+        const uint32_t w = s.index[bucket * 32 + lane];
+        const uint32_t hit = __ballot_sync(CB_FULL, w == word);
+        const uint32_t empties = __ballot_sync(CB_FULL, w == CB_IDX_EMPTY);
+        if (hit) {
+            // A bucket that still has an empty slot is the end of every probe path through it, so the
+            // slot can simply become empty again; otherwise later buckets may hold keys that probed
+            // past this one and the slot must stay marked as deleted.
+            if (lane == __ffs(hit) - 1) s.index[bucket * 32 + lane] = empties ? CB_IDX_EMPTY : CB_IDX_TOMB;
+            __syncwarp();
+            return eid;
+        }
+        if (empties) break;
+        bucket = (bucket + 1) & (nb - 1);
+    }
+    if (lane == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_PROBE_LIMIT);   // index and entries disagree
+    return eid;
+}
+
+struct TblCounters { uint32_t inserts, levict, fevict, maxprobe; };
+
+// One insertion (Section 3.1). mykey = leader[lane] (lane < LL), myfol = follower[lane] (lane < FL).
+__device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int32_t myfol, uint32_t& clock,
+                           uint32_t& count, int lane, uint32_t* status, TblCounters& cnt) {
+    const uint32_t c = ++clock;
+    cnt.inserts++;
+    const uint64_t h = warp_hash(t, mykey);
+    Probe pr = tbl_find(t, s, mykey, h, lane);
+    cnt.maxprobe = max(cnt.maxprobe, pr.probes);
+    if (pr.eid >= 0) {
+        uint32_t* e = s.entries + (size_t)pr.eid * t.E;
+        if (lane == 0) s.lstamp[pr.eid] = c;
+        const bool mine = lane < t.FC;
+        const uint32_t fs = mine ? e[t.LL + lane] : 0u;
+        bool match = mine && fs != 0u;
+        for (int j = 0; j < t.FL; ++j) {
+            const int32_t fj = __shfl_sync(CB_FULL, myfol, j);
+            if (mine && fs != 0u) match = match && ((int32_t)e[t.LL + t.FC + lane * t.FL + j] == fj);
+        }
+        const uint32_t mm = __ballot_sync(CB_FULL, match);
+        if (mm) {
+            if (t.refresh && lane == __ffs(mm) - 1) e[t.LL + lane] = c;
+        } else {
+            const uint32_t freem = __ballot_sync(CB_FULL, mine && fs == 0u);
+            int tgt;
+            if (freem) {
+                tgt = __ffs(freem) - 1;
+            } else {
+                const uint32_t g = __reduce_min_sync(CB_FULL, mine ? fs : 0xFFFFFFFFu);
+                tgt = __ffs(__ballot_sync(CB_FULL, mine && fs == g)) - 1;
+                cnt.fevict++;
+            }
+            if (lane < t.FL) e[t.LL + t.FC + tgt * t.FL + lane] = (uint32_t)myfol;
+            if (lane == 0) e[t.LL + tgt] = c;
+        }
+    } else if (pr.eid == -1) {
+        int eid;
+        if (count < (uint32_t)t.LC) {
+            eid = (int)count++;
+        } else {
+            eid = tbl_evict_lru(t, s, lane, status);
+            cnt.levict++;
+            pr = tbl_find(t, s, mykey, h, lane);           // the eviction may have opened a nearer slot
+        }
+        if (pr.free_slot == 0xFFFFFFFFu) {
+            if (lane == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_PROBE_LIMIT);
+        } else {
+            uint32_t* e = s.entries + (size_t)eid * t.E;
+            if (lane < t.LL) e[lane] = (uint32_t)mykey;
+            if (lane < t.FC) e[t.LL + lane] = lane == 0 ? c : 0u;
+            if (lane < t.FL) e[t.LL + t.FC + lane] = (uint32_t)myfol;
+            if (lane == 0) {
+                s.lstamp[eid] = c;
+                s.index[pr.free_slot] = (cb_hash_tag(h) << CB_EID_BITS) | (uint32_t)eid;
+            }
+        }
+    } else {
+        if (lane == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_PROBE_LIMIT);
+    }
+    __syncwarp();
+}
+
+// One warp per sequence; windows are applied in increasing position.
+__global__ void __launch_bounds__(128) cb_update_kernel(CbTables t, int B, const int32_t* __restrict__ tokens,
+                                                        int64_t row_stride, const int32_t* __restrict__ n_old,
+                                                        const int32_t* __restrict__ n_new, uint32_t* status,
+                                                        unsigned long long* counters) {
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (b >= B) return;
+    const CbSeq s = cb_seq(t, b);
+    const int w = t.LL + t.FL;
+    const int n0 = n_old[b], n1 = n_new[b];
+    uint32_t clock = s.hdr[0], count = s.hdr[1];
+    TblCounters cnt = {0, 0, 0, 0};
+    const int32_t* row = tokens + (size_t)b * row_stride;
+    for (int i = max(0, n0 - w + 1); i + w <= n1; ++i) {
+        const int32_t mykey = lane < t.LL ? row[i + lane] : 0;
+        const int32_t myfol = lane < t.FL ? row[i + t.LL + lane] : 0;
+        tbl_insert(t, s, mykey, myfol, clock, count, lane, status, cnt);
+    }
+    if (lane == 0) {
+        s.hdr[0] = clock; s.hdr[1] = count;
+        if (cnt.inserts) atomicAdd(&counters[CB_CNT_INSERTS], (unsigned long long)cnt.inserts);
+        if (cnt.levict) atomicAdd(&counters[CB_CNT_LEADER_EVICTIONS], (unsigned long long)cnt.levict);
+        if (cnt.fevict) atomicAdd(&counters[CB_CNT_FOLLOWER_EVICTIONS], (unsigned long long)cnt.fevict);
+        if (cnt.maxprobe) atomicMax(&counters[CB_CNT_MAX_PROBE], (unsigned long long)cnt.maxprobe);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Draft-tree expansion: one CTA per sequence, one warp per frontier leaf ("branch") for the lookups.
+// Each level: (1) warps look up the keys of all frontier leaves in parallel and stage the followers,
+// most recent first, in shared memory; (2) one thread replays the sequential breadth-first order over
+// the staged results, which fixes node indices, the point where the size cap ends the level and the
+// ordinal of every query that the sequential order would have issued; (3) the leaders of those queries
+// get their new recency stamp with an atomic max (two leaves of one level may share a leader).
+struct DraftSmem {
+    int32_t* tok; int32_t* par; int32_t* dep;
+    int32_t* front; int32_t* next;
+    int32_t* r_eid; int32_t* r_nf; int32_t* r_ok; uint32_t* r_stamp;
+    int32_t* fol;
+};
+
+__global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, int T, int crt, int max_depth, int NL,
+                                                       const int32_t* __restrict__ tokens, int64_t row_stride,
+                                                       const int32_t* __restrict__ seq_len,
+                                                       int32_t* __restrict__ o_tok, int32_t* __restrict__ o_par,
+                                                       int32_t* __restrict__ o_dep, uint32_t* __restrict__ o_mask,
+                                                       int32_t* __restrict__ o_n, uint32_t* status,
+                                                       unsigned long long* counters) {
+    extern __shared__ int32_t smem[];
+    DraftSmem S;
+    S.tok = smem; S.par = S.tok + T; S.dep = S.par + T;
+    S.front = S.dep + T; S.next = S.front + NL;
+    S.r_eid = S.next + NL; S.r_nf = S.r_eid + NL; S.r_ok = S.r_nf + NL; S.r_stamp = (uint32_t*)(S.r_ok + NL);
+    S.fol = (int32_t*)(S.r_stamp + NL);
+    __shared__ int sh_n, sh_nfront, sh_nnext, sh_q, sh_hits, sh_level;
+
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    const CbSeq s = cb_seq(t, b);
+    const int32_t* row = tokens + (size_t)b * row_stride;
+    const int L = seq_len[b];
+    const int W = (T + 31) >> 5;
+    const int FLFC = t.FL * t.FC;
+    const uint32_t clock0 = s.hdr[0];
+
+    for (int i = tid; i < T; i += blockDim.x) { S.tok[i] = -1; S.par[i] = -1; S.dep[i] = -1; }
+    if (tid == 0) {
+        sh_n = 0; sh_nfront = 0; sh_q = 0; sh_hits = 0; sh_level = 1;
+    }
+    __syncthreads();
+    if (tid == 0 && L >= 1) {
+        S.tok[0] = row[L - 1]; S.dep[0] = 0; sh_n = 1; S.front[0] = 0; sh_nfront = 1;
+    }
+    __syncthreads();
+
+    while (true) {
+        const int nfront = sh_nfront, n_now = sh_n;
+        if (nfront == 0 || n_now >= T) break;
+        // (1) parallel lookups, one warp per leaf
+        for (int li = warp; li < nfront; li += nwarps) {
+            const int leaf = S.front[li];
+            const int d = S.dep[leaf];
+            // key = last LL tokens of (row[0 .. L-1) ++ root->leaf path); lane j < LL holds key[j]
+            int32_t mykey = 0;
+            bool ok = d < max_depth;
+            if (lane < t.LL) {
+                const int back = t.LL - 1 - lane;         // distance from the leaf along the sequence
+                if (back <= d) {
+                    int c = leaf;
+                    for (int k = 0; k < back; ++k) c = S.par[c];
+                    mykey = S.tok[c];
+                } else {
+                    const int pos = L - 1 - (back - d);
+                    mykey = pos >= 0 ? row[pos] : -1;
+                }
+            }
+            ok = ok && __all_sync(CB_FULL, mykey >= 0);
+            int eid = -1, nf = 0;
+            if (ok) {
+                const uint64_t h = warp_hash(t, mykey);
+                const Probe pr = tbl_find(t, s, mykey, h, lane);
+                if (pr.eid == -2 && lane == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_PROBE_LIMIT);
+                if (pr.eid >= 0) {
+                    eid = pr.eid;
+                    const uint32_t* e = s.entries + (size_t)eid * t.E;
+                    const uint32_t fs = lane < t.FC ? e[t.LL + lane] : 0u;
+                    // rank = number of followers inserted more recently than mine (stamps are unique)
+                    int rank = 0;
+                    for (int f = 0; f < t.FC; ++f) {
+                        const uint32_t o = __shfl_sync(CB_FULL, fs, f);
+                        rank += (o > fs) ? 1 : 0;
+                    }
+                    nf = __popc(__ballot_sync(CB_FULL, fs != 0u));
+                    if (lane < t.FC && fs != 0u)
+                        for (int j = 0; j < t.FL; ++j)
+                            S.fol[li * FLFC + rank * t.FL + j] = (int32_t)e[t.LL + t.FC + lane * t.FL + j];
+                }
+            }
+            if (lane == 0) { S.r_eid[li] = eid; S.r_nf[li] = nf; S.r_ok[li] = ok ? 1 : 0; S.r_stamp[li] = 0u; }
+        }
+        __syncthreads();
+        // (2) sequential replay of the breadth-first order
+        if (tid == 0) {
+            int n = n_now, q = sh_q, hits = sh_hits, nn = 0;
+            const int cap = (sh_level == 1) ? max(1, T - crt) : T;
+            for (int li = 0; li < nfront; ++li) {
+                if (n >= cap) break;
+                if (!S.r_ok[li]) continue;
+                ++q;                                            // this query is issued: the clock ticks
+                if (S.r_eid[li] < 0) continue;
+                ++hits;
+                S.r_stamp[li] = clock0 + (uint32_t)q;
+                const int leaf = S.front[li];
+                for (int f = 0; f < S.r_nf[li]; ++f) {
+                    if (n >= cap) break;
+                    int p = leaf, k = 0;
+                    for (int j = 0; j < t.FL; ++j) {
+                        if (n >= cap || S.dep[p] >= max_depth) break;
+                        S.tok[n] = S.fol[li * FLFC + f * t.FL + j];
+                        S.par[n] = p; S.dep[n] = S.dep[p] + 1; p = n; ++n; ++k;
+                    }
+                    if (k == t.FL) S.next[nn++] = p;
+                }
+            }
+            sh_n = n; sh_q = q; sh_hits = hits; sh_nnext = nn; sh_level = sh_level + 1;
+        }
+        __syncthreads();
+        // (3) stamp the leaders the sequential order reached; publish the next frontier
+        for (int li = tid; li < nfront; li += blockDim.x)
+            if (S.r_stamp[li] != 0u) atomicMax(&s.lstamp[S.r_eid[li]], S.r_stamp[li]);
+        const int nn = sh_nnext;
+        __syncthreads();
+        for (int i = tid; i < nn; i += blockDim.x) S.front[i] = S.next[i];
+        if (tid == 0) sh_nfront = nn;
+        __syncthreads();
+    }
+
+    const int n = sh_n;
+    if (tid == 0) {
+        s.hdr[0] = clock0 + (uint32_t)sh_q;
+        o_n[b] = n;
+        if (sh_q) atomicAdd(&counters[CB_CNT_QUERIES], (unsigned long long)sh_q);
+        if (sh_hits) atomicAdd(&counters[CB_CNT_QUERY_HITS], (unsigned long long)sh_hits);
+    }
+    for (int i = tid; i < T; i += blockDim.x) {
+        o_tok[(size_t)b * T + i] = S.tok[i];
+        o_par[(size_t)b * T + i] = S.par[i];
+        o_dep[(size_t)b * T + i] = S.dep[i];
+        uint32_t m[4] = {0u, 0u, 0u, 0u};
+        if (i < n) for (int c = i; c >= 0; c = S.par[c]) m[c >> 5] |= 1u << (c & 31);
+        for (int k = 0; k < W; ++k) o_mask[((size_t)b * T + i) * W + k] = m[k];
+    }
+}
+
+}  // namespace
+
+extern "C" cb_status cb_update(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* n_old,
+                               const int32_t* n_new, void* stream) {
+    CB_CHECK_ARG(ctx && tokens && n_old && n_new && row_stride >= 1);
+    const int B = ctx->cfg.batch, wpb = 4;
+    cb_update_kernel<<<(B + wpb - 1) / wpb, wpb * 32, 0, (cudaStream_t)stream>>>(
+        ctx->tables, B, tokens, row_stride, n_old, n_new, ctx->d_status, ctx->d_counters);
+    cb_count_launch(1);
+    CB_CUDA(cudaGetLastError());
+    return CB_OK;
+}
+
+extern "C" cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* seq_len,
+                                   int32_t* tree_tokens, int32_t* tree_parent, int32_t* tree_depth,
+                                   uint32_t* tree_mask, int32_t* n_nodes, void* stream) {
+    CB_CHECK_ARG(ctx && tokens && seq_len && tree_tokens && tree_parent && tree_depth && tree_mask && n_nodes);
+    CB_CHECK_ARG(row_stride >= 1);
+    const cb_config& c = ctx->cfg;
+    const int T = c.max_nodes;
+    const int NL = min(T, (T - 1) / c.FL + 1);
+    const size_t smem = sizeof(int32_t) * ((size_t)3 * T + (size_t)6 * NL + (size_t)NL * c.FL * c.FC);
+    if (smem > 48 * 1024) return CB_ERR_UNSUPPORTED;
+    const int threads = 32 * max(1, min(8, NL));
+    cb_draft_kernel<<<c.batch, threads, smem, (cudaStream_t)stream>>>(
+        ctx->tables, T, c.crt, c.max_depth, NL, tokens, row_stride, seq_len, tree_tokens, tree_parent,
+        tree_depth, tree_mask, n_nodes, ctx->d_status, ctx->d_counters);
+    cb_count_launch(1);
+    CB_CUDA(cudaGetLastError());
+    return CB_OK;
+}

@@ -1,0 +1,46 @@
+"""Device-side fills (workloads/fill.cu): the same tensors as rng.py, produced on the GPU."""
+import ctypes as C
+import os
+import subprocess
+
+import torch
+
+from .rng import stream_key, NORMAL_SCALE_F32
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fill.cu")
+_SO = os.path.join(_HERE, "libcbfill.so")
+_lib = None
+
+
+def build(force=False):
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+        tmp = _SO + ".tmp%d" % os.getpid()
+        subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-shared",
+                               "-Xcompiler", "-fPIC", "-o", tmp, _SRC])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.wl_fill_normal.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, C.c_float, C.c_int, C.c_void_p]
+        _lib.wl_fill_normal.restype = C.c_int
+    return _lib
+
+
+def fill_normal(t: torch.Tensor, seed: int, tid: int):
+    """In-place: t.flatten()[i] = normal(seed, tid, i); t is a contiguous CUDA tensor, bf16 or float32."""
+    assert t.is_cuda and t.is_contiguous() and t.dtype in (torch.bfloat16, torch.float32)
+    rc = _load().wl_fill_normal(t.data_ptr(), t.numel(), stream_key(seed, tid), float(NORMAL_SCALE_F32),
+                                int(t.dtype == torch.bfloat16), torch.cuda.current_stream().cuda_stream)
+    if rc != 0:
+        raise RuntimeError("wl_fill_normal failed with CUDA error %d" % rc)
+    return t
+
+
+def normal_tensor(shape, dtype, seed, tid, device="cuda:0"):
+    return fill_normal(torch.empty(shape, dtype=dtype, device=device), seed, tid)

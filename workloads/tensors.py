@@ -60,6 +60,22 @@ def pool_full_bits(cfg: CbConfig, num_pages: int):
             normal_bf16_bits(cfg.seed, TID.V_POOL, idx).reshape(shape))
 
 
+def pool_pages_bits(cfg: CbConfig, pages: np.ndarray):
+    """The given pages of the pool, all kv heads, as bf16 bit patterns [len(pages), P, Hkv, D] for K and V."""
+    P, H, D = cfg.page_size, cfg.n_kv_heads, cfg.head_dim
+    per = P * H * D
+    idx = np.asarray(pages, dtype=np.int64)[:, None] * per + np.arange(per)[None, :]
+    shape = (len(pages), P, H, D)
+    return (normal_bf16_bits(cfg.seed, TID.K_POOL, idx).reshape(shape),
+            normal_bf16_bits(cfg.seed, TID.V_POOL, idx).reshape(shape))
+
+
+def seq_bits(cfg: CbConfig, tid: int, b: int, heads: int):
+    """One sequence's slice of a [B, T, heads, D] tensor as bf16 bit patterns [T, heads, D]."""
+    per = cfg.max_nodes * heads * cfg.head_dim
+    return normal_bf16_bits(cfg.seed, tid, b * per + np.arange(per)).reshape(cfg.max_nodes, heads, cfg.head_dim)
+
+
 def tree_kv(cfg: CbConfig, b: int, kv_head: int, as_f32=True):
     """K and V of the draft-tree tokens of sequence b, one kv head: layout [B, T, Hkv, D] -> [T, D]."""
     T, H, D = cfg.max_nodes, cfg.n_kv_heads, cfg.head_dim
