@@ -44,7 +44,8 @@ typedef enum {
     CB_ERR_CUDA = 3,
     CB_ERR_PROBE_LIMIT = 4, /* device: a hash probe visited every bucket without finding a free slot  */
     CB_ERR_TIMEOUT = 5,     /* device: a bounded wait (mbarrier / flag) ran out                        */
-    CB_ERR_UNSUPPORTED = 6
+    CB_ERR_UNSUPPORTED = 6,
+    CB_ERR_STATIC_LIMIT = 7 /* cb_accept_static: the problem does not fit the built-in scratch array        */
 } cb_status;
 
 enum { CB_DTYPE_F32 = 0, CB_DTYPE_BF16 = 1 };
@@ -187,6 +188,38 @@ cb_status cb_accept(cb_ctx* ctx, const int32_t* tree_tokens, const int32_t* tree
                     int32_t logits_dtype, int64_t logits_row_stride, const int32_t* target_ids_in,
                     int32_t* n_accept, int32_t* accept_nodes, int32_t* out_tokens,
                     int32_t* target_ids_out, void* stream);
+
+/*
+ * cb_accept_static — cb_accept (logits form) for callers that must not allocate device memory.
+ * (The paper has no counterpart; this is a packaging variant of the call above.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits — inside a framework's memory pool whose
+ * owner forbids side allocations, in a plugin that is handed buffers but no allocator, or under a
+ * memory budget that is fixed before the library is loaded.  Such a caller cannot provide the workspace
+ * cb_create wants, so this entry point needs no context at all: the scratch that the arg-max reduction
+ * uses (one packed maximum per logits row and one arrival counter per sequence) lives in a fixed array
+ * that is part of the library image.  Every GPU that loads the library carries that array
+ * (CB_STATIC_MAX_ROWS * 8 + CB_STATIC_MAX_BATCH * 4 bytes = 68 KiB) until the process exits.
+ *
+ * Shape arguments replace the context: batch, max_nodes (1..128), max_depth (>= 0), vocab (>= 1).
+ * All other arguments, the result and the tie rules are exactly those of cb_accept with logits given;
+ * target_ids_out may be NULL.
+ *
+ * Limits: batch <= CB_STATIC_MAX_BATCH and batch * max_nodes <= CB_STATIC_MAX_ROWS; anything larger
+ * returns CB_ERR_STATIC_LIMIT and enqueues nothing.
+ *
+ * The call never allocates or frees (no cudaMalloc / cudaFree, no allocating library routine).  The first
+ * call on each device looks up the array's device address once, with that device current; make that
+ * first call outside any stream capture.  Before each launch the part of the array in use is cleared
+ * on `stream`.  All calls on a device share the one array: two calls that may overlap on the GPU
+ * (different streams without an ordering between them) race on it and give wrong results; order them.
+ */
+enum { CB_STATIC_MAX_BATCH = 1024, CB_STATIC_MAX_ROWS = 8192 };
+cb_status cb_accept_static(int32_t batch, int32_t max_nodes, int32_t max_depth, int32_t vocab,
+                           const int32_t* tree_tokens, const int32_t* tree_parent, const int32_t* tree_depth,
+                           const int32_t* n_nodes, const void* logits, int32_t logits_dtype,
+                           int64_t logits_row_stride, int32_t* n_accept, int32_t* accept_nodes,
+                           int32_t* out_tokens, int32_t* target_ids_out, void* stream);
 
 /*
  * Canonical view of one sequence's table, for checkpointing and for comparing table contents:

@@ -9,12 +9,14 @@ SO_PATH = os.path.join(HERE, "libcacheback.so")
 CB_OK = 0
 CB_DTYPE_F32, CB_DTYPE_BF16 = 0, 1
 CB_FLAG_NO_FOLLOWER_REFRESH, CB_FLAG_ATTN_CUDA_CORES = 1, 2
+CB_ERR_STATIC_LIMIT = 7
+CB_STATIC_MAX_BATCH, CB_STATIC_MAX_ROWS = 1024, 8192
 CB_NUM_COUNTERS = 8
 COUNTER_NAMES = ["inserts", "leader_evictions", "follower_evictions", "queries", "query_hits", "max_probe"]
 
 EXPORTS = ["cb_workspace_bytes", "cb_create", "cb_destroy", "cb_reset", "cb_update", "cb_draft_tree",
            "cb_tree_attn", "cb_accept", "cb_table_dump", "cb_table_load", "cb_poll_status", "cb_launch_count",
-           "cb_status_str"]
+           "cb_status_str", "cb_accept_static"]
 
 
 class CbConfigC(C.Structure):
@@ -49,6 +51,7 @@ def load():
     L.cb_draft_tree.argtypes = [vp, vp, i64, vp, vp, vp, vp, vp, vp, vp]
     L.cb_tree_attn.argtypes = [vp, C.POINTER(CbAttnArgsC), vp]
     L.cb_accept.argtypes = [vp, vp, vp, vp, vp, vp, i32, i64, vp, vp, vp, vp, vp, vp]
+    L.cb_accept_static.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, i64, vp, vp, vp, vp, vp]
     L.cb_table_dump.argtypes = [vp, i32, C.POINTER(i32), vp, vp, vp]
     L.cb_table_load.argtypes = [vp, i32, i32, vp, vp, vp]
     L.cb_poll_status.argtypes = [vp, C.POINTER(i32), vp]

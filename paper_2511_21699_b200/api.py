@@ -35,6 +35,36 @@ def _stream(stream):
     return (stream if stream is not None else torch.cuda.current_stream()).cuda_stream
 
 
+def cb_accept_static(tree, logits, max_depth, res=None, stream=None):
+    """Greedy acceptance from logits without a context and without any device allocation by the library:
+    for callers that only have the buffers they were given (a plugin inside someone else's memory pool, a
+    fixed memory budget).  The library's built-in scratch array is used instead of a workspace, so batch is
+    limited to 1,024 and batch * max_nodes to 8,192; larger shapes raise CachebackError.  Calls on one device
+    share that array: do not let two of them overlap on the GPU.  Make the first call on a device outside
+    any stream capture.  `res` holds the caller-allocated outputs (n_accept [B], accept_nodes [B, max_depth],
+    out_tokens [B, max_depth + 1], target_ids [B, T]); it is created with torch when omitted."""
+    lib = _lib.load()
+    B, T, V = logits.shape
+    if logits.dtype == torch.float32:
+        dtype = _lib.CB_DTYPE_F32
+    elif logits.dtype == torch.bfloat16:
+        dtype = _lib.CB_DTYPE_BF16
+    else:
+        raise CachebackError("logits must be float32 or bfloat16")
+    if not (logits.is_cuda and logits.stride(2) == 1 and logits.stride(0) == T * logits.stride(1)):
+        raise CachebackError("logits must be [batch, max_nodes, vocab] with a uniform row stride")
+    if res is None:
+        i32 = dict(dtype=torch.int32, device=logits.device)
+        res = dict(n_accept=torch.empty(B, **i32), accept_nodes=torch.empty(B, max_depth, **i32),
+                   out_tokens=torch.empty(B, max_depth + 1, **i32), target_ids=torch.empty(B, T, **i32))
+    _check(lib.cb_accept_static(B, T, max_depth, V, _ptr(tree["tokens"], torch.int32), _ptr(tree["parent"], torch.int32),
+                                _ptr(tree["depth"], torch.int32), _ptr(tree["n_nodes"], torch.int32), logits.data_ptr(), dtype,
+                                logits.stride(1), _ptr(res["n_accept"], torch.int32), _ptr(res["accept_nodes"], torch.int32),
+                                _ptr(res["out_tokens"], torch.int32), _ptr(res["target_ids"], torch.int32), _stream(stream)),
+           "cb_accept_static")
+    return res
+
+
 class Cacheback:
     """One context: per-sequence tables plus scratch, in a workspace tensor owned by this object."""
 

@@ -238,3 +238,83 @@ extern "C" cb_status cb_accept(cb_ctx* ctx, const int32_t* tree_tokens, const in
     CB_CUDA(cudaGetLastError());
     return CB_OK;
 }
+
+// ---------------------------------------------------------------------------------------------------
+// cb_accept_static: the logits form of cb_accept for callers that are not allowed to allocate device
+// memory (no workspace, no context).  Its scratch is this file-scope array, part of the library image:
+// [0, CB_STATIC_MAX_ROWS) packed row maxima (8 bytes each), then CB_STATIC_MAX_BATCH arrival counters.
+// In host code the name g_static_scratch is only a handle for cudaGetSymbolAddress, never a device
+// pointer; the per-device address is looked up once and handed to the kernel as an ordinary argument.
+#include <mutex>
+
+static __device__ __align__(256) unsigned long long g_static_scratch[CB_STATIC_MAX_ROWS + CB_STATIC_MAX_BATCH / 2];
+
+namespace {
+constexpr int kMaxDevices = 64;
+struct StaticSetup { unsigned long long* rowmax; uint32_t* ticket; int num_sms; bool ready; };
+StaticSetup g_setup[kMaxDevices];
+std::mutex g_setup_mutex;
+
+// One-time set-up for the current device: resolve the array's device address and read the SM count.
+cb_status static_setup(int dev, StaticSetup* out) {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    StaticSetup& s = g_setup[dev];
+    if (!s.ready) {
+        void* ptr = nullptr;
+        CB_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        int sms = 0;
+        CB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        s.rowmax = (unsigned long long*)ptr;
+        s.ticket = (uint32_t*)(s.rowmax + CB_STATIC_MAX_ROWS);
+        s.num_sms = sms;
+        s.ready = true;
+    }
+    *out = s;
+    return CB_OK;
+}
+}  // namespace
+
+extern "C" cb_status cb_accept_static(int32_t batch, int32_t max_nodes, int32_t max_depth, int32_t vocab,
+                                      const int32_t* tree_tokens, const int32_t* tree_parent, const int32_t* tree_depth,
+                                      const int32_t* n_nodes, const void* logits, int32_t logits_dtype,
+                                      int64_t logits_row_stride, int32_t* n_accept, int32_t* accept_nodes,
+                                      int32_t* out_tokens, int32_t* target_ids_out, void* stream) {
+    CB_CHECK_ARG(tree_tokens && tree_parent && tree_depth && n_nodes && logits && n_accept && accept_nodes && out_tokens);
+    CB_CHECK_ARG(batch >= 1 && max_nodes >= 1 && max_nodes <= CB_MAX_T && max_depth >= 0 && vocab >= 1);
+    CB_CHECK_ARG(logits_dtype == CB_DTYPE_F32 || logits_dtype == CB_DTYPE_BF16);
+    CB_CHECK_ARG(logits_row_stride >= vocab);
+    const int esz = logits_dtype == CB_DTYPE_F32 ? 4 : 2;
+    CB_CHECK_ARG(((uintptr_t)logits & (esz - 1)) == 0);
+    if (batch > CB_STATIC_MAX_BATCH || (long)batch * max_nodes > CB_STATIC_MAX_ROWS) {
+        fprintf(stderr, "cacheback: cb_accept_static: batch %d x max_nodes %d exceeds the built-in scratch "
+                        "(batch <= %d, batch * max_nodes <= %d)\n", batch, max_nodes, CB_STATIC_MAX_BATCH, CB_STATIC_MAX_ROWS);
+        return CB_ERR_STATIC_LIMIT;
+    }
+    int dev = 0;
+    CB_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CB_ERR_UNSUPPORTED;
+    StaticSetup su;
+    const cb_status ss = static_setup(dev, &su);
+    if (ss != CB_OK) return ss;
+    cudaStream_t st = (cudaStream_t)stream;
+    // The array is shared by every call and keeps what the last one left: clear the part this call uses.
+    CB_CUDA(cudaMemsetAsync(su.rowmax, 0, (size_t)batch * max_nodes * sizeof(unsigned long long), st));
+    CB_CUDA(cudaMemsetAsync(su.ticket, 0, (size_t)batch * sizeof(uint32_t), st));
+    int chunk = 32768 / esz;
+    if ((long)batch * max_nodes >= 8L * su.num_sms) chunk *= 4;
+    int cpr = (vocab + chunk - 1) / chunk;
+    chunk = ((vocab + cpr - 1) / cpr + 7) & ~7;
+    cpr = (vocab + chunk - 1) / chunk;
+    dim3 grid(cpr, max_nodes, batch);
+    if (logits_dtype == CB_DTYPE_F32)
+        cb_accept_logits_kernel<false><<<grid, 256, 0, st>>>(max_nodes, vocab, max_depth, chunk, cpr, logits, logits_row_stride,
+                                                             tree_tokens, tree_parent, tree_depth, n_nodes, su.rowmax, su.ticket,
+                                                             n_accept, accept_nodes, out_tokens, target_ids_out);
+    else
+        cb_accept_logits_kernel<true><<<grid, 256, 0, st>>>(max_nodes, vocab, max_depth, chunk, cpr, logits, logits_row_stride,
+                                                            tree_tokens, tree_parent, tree_depth, n_nodes, su.rowmax, su.ticket,
+                                                            n_accept, accept_nodes, out_tokens, target_ids_out);
+    cb_count_launch(1);
+    CB_CUDA(cudaGetLastError());
+    return CB_OK;
+}

@@ -215,6 +215,7 @@ extern "C" const char* cb_status_str(cb_status s) {
         case CB_ERR_PROBE_LIMIT: return "hash probe limit reached";
         case CB_ERR_TIMEOUT: return "bounded device wait ran out";
         case CB_ERR_UNSUPPORTED: return "unsupported device or shape";
+        case CB_ERR_STATIC_LIMIT: return "problem larger than the built-in static scratch (see cb_accept_static)";
     }
     return "unknown status";
 }

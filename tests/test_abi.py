@@ -1,0 +1,38 @@
+"""The C-ABI library loads without a GPU and exports every function the public header declares."""
+import ctypes
+import os
+import re
+
+from tests.conftest import ROOT
+
+
+def _declared():
+    with open(os.path.join(ROOT, "include", "cacheback.h")) as f:
+        src = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
+    return sorted(set(re.findall(r"\b(cb_[a-z_0-9]+)\s*\(", src)))
+
+
+def test_header_symbols_are_exported():
+    import __graft_entry__
+    __graft_entry__.build()
+    from paper_2511_21699_b200 import _lib
+    lib = _lib.load()
+    names = _declared()
+    assert {"cb_update", "cb_draft_tree", "cb_tree_attn", "cb_accept"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(_lib.EXPORTS) == set(names)
+
+
+def test_host_side_argument_checks_need_no_gpu():
+    from paper_2511_21699_b200 import _lib
+    lib = _lib.load()
+    cfg = _lib.CbConfigC(1, 2, 3, 4096, 4, 16, 4, 5, 32000, 8, 8, 64, 16, 0)
+    n = ctypes.c_size_t(0)
+    assert lib.cb_workspace_bytes(ctypes.byref(cfg), ctypes.byref(n)) == 0 and n.value > 4096 * 4
+    bad = _lib.CbConfigC(1, 2, 3, 4096, 4, 16, 4, 5, 32000, 8, 3, 64, 16, 0)      # heads do not divide
+    assert lib.cb_workspace_bytes(ctypes.byref(bad), ctypes.byref(n)) == 1
+    bad = _lib.CbConfigC(1, 2, 3, 4096, 4, 256, 4, 5, 32000, 8, 8, 64, 16, 0)     # tree cap above 128
+    assert lib.cb_workspace_bytes(ctypes.byref(bad), ctypes.byref(n)) == 1
+    assert lib.cb_status_str(4).decode().startswith("hash probe")
+    assert lib.cb_accept_static(4096, 16, 4, 100, 1, 1, 1, 1, 8, 0, 100, 1, 1, 1, None, None) == _lib.CB_ERR_STATIC_LIMIT
