@@ -1,8 +1,8 @@
-// cb_tree_attn entry point, the split-KV combine pass and the plain CUDA-core attention kernel.
+// cb_tree_attn entry point and the plain CUDA-core attention kernel.
 //
 // The CUDA-core kernel is a debugging aid (CB_FLAG_ATTN_CUDA_CORES): four threads per query row, fp32
-// dot products from bf16 tiles staged in shared memory, one online-softmax update per key.  The
-// production path is the tensor-core kernel in cb_attn_tc.cu; both write the same partial format.
+// dot products from bf16 tiles staged in shared memory, one online-softmax update per key, one CTA per
+// (row tile, sequence, kv head).  The production path is the tensor-core kernel in cb_attn_tc.cu.
 #include <math.h>
 
 #include "cb_attn.cuh"
@@ -15,7 +15,7 @@ __global__ void __launch_bounds__(512) cb_attn_cc_kernel(CbAttnParams p) {
     constexpr int DQ = D / 4;
     __shared__ __align__(16) __nv_bfloat16 Ks[32][D];
     __shared__ __align__(16) __nv_bfloat16 Vs[32][D];
-    const int split = blockIdx.x, mt = blockIdx.y, bk = blockIdx.z;
+    const int mt = blockIdx.y, bk = blockIdx.z;
     const int b = bk / p.Hkv, kh = bk % p.Hkv;
     const int tid = threadIdx.x, rl = tid >> 2, qd = tid & 3;
     const int n = p.n_nodes[b], ctx = p.ctx_len[b];
@@ -34,10 +34,8 @@ __global__ void __launch_bounds__(512) cb_attn_cc_kernel(CbAttnParams p) {
     uint32_t mrow[4] = {0u, 0u, 0u, 0u};
     if (valid) for (int k = 0; k < p.W; ++k) mrow[k] = p.tree_mask[((size_t)b * p.T + i) * p.W + k];
 
-    int t_lo, t_hi;
-    cb_split_range(ctx, p.nsplit, split, &t_lo, &t_hi);
     const int nct = (ctx + CB_KT - 1) / CB_KT;
-    for (int tile = t_lo; tile < t_hi; ++tile) {
+    for (int tile = 0; tile <= nct; ++tile) {
         const bool is_tree = tile == nct;
         const int kbase = is_tree ? 0 : tile * CB_KT;
         const int klim = is_tree ? n : ctx;
@@ -100,80 +98,22 @@ __global__ void __launch_bounds__(512) cb_attn_cc_kernel(CbAttnParams p) {
         }
     }
 
-    if (p.nsplit == 1) {
-        if (exists) {
-            const int io = node, ho = kh * p.G + rl % p.G;
-            __nv_bfloat16* op = p.out + (((size_t)b * p.T + io) * p.Hq + ho) * D + qd * DQ;
-            const float inv = (valid && l > 0.f) ? 1.f / l : 0.f;
+    if (exists) {
+        const int io = node, ho = kh * p.G + rl % p.G;
+        __nv_bfloat16* op = p.out + (((size_t)b * p.T + io) * p.Hq + ho) * D + qd * DQ;
+        const float inv = (valid && l > 0.f) ? 1.f / l : 0.f;
 #pragma unroll
-            for (int d = 0; d < DQ; ++d) op[d] = __float2bfloat16_rn(acc[d] * inv);
-            if (p.lse && qd == 0) p.lse[((size_t)b * p.Hq + ho) * p.T + io] = (valid && l > 0.f) ? (m + log2f(l)) * 0.6931471805599453f : 0.f;
-        }
-    } else {
-        const size_t slot = ((size_t)bk * p.MT + mt) * p.nsplit + split;
-        float* pp = p.part + (slot * CB_MT + rl) * (D + 4);
-#pragma unroll
-        for (int d = 0; d < DQ; ++d) pp[qd * DQ + d] = acc[d];
-        if (qd == 0) { pp[D] = m; pp[D + 1] = l; }
+        for (int d = 0; d < DQ; ++d) op[d] = __float2bfloat16_rn(acc[d] * inv);
+        if (p.lse && qd == 0) p.lse[((size_t)b * p.Hq + ho) * p.T + io] = (valid && l > 0.f) ? (m + log2f(l)) * 0.6931471805599453f : 0.f;
     }
-}
-
-// ---------------------------------------------------------------------------------------------------
-// Combine: one warp per output row; merges the nsplit partials of its unit.
-template <int D>
-__global__ void __launch_bounds__(256) cb_attn_combine_kernel(CbAttnParams p) {
-    const int lane = threadIdx.x & 31;
-    const long row = (long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // over B * Hkv * G * T
-    const long rows_per_unit = (long)p.G * p.T;
-    if (row >= (long)p.B * p.Hkv * rows_per_unit) return;
-    const int bk = (int)(row / rows_per_unit), r = (int)(row % rows_per_unit);
-    const int b = bk / p.Hkv, kh = bk % p.Hkv;
-    const int i = r / p.G, h = kh * p.G + r % p.G;
-    const int mt = i / p.NPT, rl = (i % p.NPT) * p.G + r % p.G;
-    const int n = p.n_nodes[b];
-    constexpr int PER = D / 32;
-    float o[PER];
-#pragma unroll
-    for (int d = 0; d < PER; ++d) o[d] = 0.f;
-    float M = -INFINITY, Lsum = 0.f;
-    if (i < n) {
-        const float* base = p.part + (((size_t)bk * p.MT + mt) * p.nsplit * CB_MT + rl) * (D + 4);
-        const size_t sstride = (size_t)CB_MT * (D + 4);
-        for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, base[s * sstride + D]);
-        for (int s = 0; s < p.nsplit; ++s) {
-            const float* pp = base + s * sstride;
-            const float ms = pp[D];
-            if (ms == -INFINITY) continue;
-            const float w = exp2f(ms - M);
-            Lsum += w * pp[D + 1];
-#pragma unroll
-            for (int d = 0; d < PER; ++d) o[d] = fmaf(w, pp[lane * PER + d], o[d]);
-        }
-    }
-    const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
-    __nv_bfloat16* op = p.out + (((size_t)b * p.T + i) * p.Hq + h) * D + lane * PER;
-#pragma unroll
-    for (int d = 0; d < PER; ++d) op[d] = __float2bfloat16_rn(o[d] * inv);
-    if (p.lse && lane == 0) p.lse[((size_t)b * p.Hq + h) * p.T + i] = Lsum > 0.f ? (M + log2f(Lsum)) * 0.6931471805599453f : 0.f;
 }
 
 }  // namespace
 
 cb_status cb_attn_launch_cuda_cores(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t st) {
-    dim3 grid(p.nsplit, p.MT, p.B * p.Hkv);
+    dim3 grid(1, p.MT, p.B * p.Hkv);
     if (p.D == 128) cb_attn_cc_kernel<128><<<grid, 512, 0, st>>>(p);
     else cb_attn_cc_kernel<64><<<grid, 512, 0, st>>>(p);
-    cb_count_launch(1);
-    CB_CUDA(cudaGetLastError());
-    return CB_OK;
-}
-
-cb_status cb_attn_launch_combine(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t st) {
-    const long rows = (long)p.B * p.Hkv * p.G * p.T;
-    const int wpb = 8;
-    const unsigned grid = (unsigned)((rows + wpb - 1) / wpb);
-    if (p.D == 128) cb_attn_combine_kernel<128><<<grid, wpb * 32, 0, st>>>(p);
-    else cb_attn_combine_kernel<64><<<grid, wpb * 32, 0, st>>>(p);
     cb_count_launch(1);
     CB_CUDA(cudaGetLastError());
     return CB_OK;
@@ -202,24 +142,9 @@ extern "C" cb_status cb_tree_attn(cb_ctx* ctx, const cb_attn_args* a, void* stre
     const float scale = a->scale > 0.f ? a->scale : 1.0f / sqrtf((float)c.head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = ctx->d_status;
-    // Split the keys of one (sequence, kv head, row tile) over several CTAs when the units alone cannot
-    // fill the machine; partials are merged by the combine pass.
-    const int max_ctx = a->max_ctx > 0 ? a->max_ctx : a->max_pages * c.page_size;
-    const int max_tiles = (max_ctx + CB_KT - 1) / CB_KT + 1;
-    const long units = (long)p.B * p.Hkv * p.MT;
-    int nsplit = 1;
-    if (units < 2L * ctx->num_sms) {
-        nsplit = (int)((2L * ctx->num_sms + units - 1) / units);
-        nsplit = (int)fminf((float)nsplit, (float)max_tiles);
-        nsplit = (int)fminf((float)nsplit, (float)(ctx->attn_max_units / units));
-        if (nsplit < 1) nsplit = 1;
-    }
-    p.nsplit = nsplit;
+    // The tensor-core kernel is persistent: one CTA per SM, each taking an equal share of all key tiles.
+    p.nc = ctx->num_sms < CB_ATTN_MAX_CTAS ? ctx->num_sms : CB_ATTN_MAX_CTAS;
     cudaStream_t st = (cudaStream_t)stream;
-    cb_status s;
-    if (c.flags & CB_FLAG_ATTN_CUDA_CORES) s = cb_attn_launch_cuda_cores(ctx, p, st);
-    else s = cb_attn_launch_tensor(ctx, p, st);
-    if (s != CB_OK) return s;
-    if (nsplit > 1) s = cb_attn_launch_combine(ctx, p, st);
-    return s;
+    if (c.flags & CB_FLAG_ATTN_CUDA_CORES) return cb_attn_launch_cuda_cores(ctx, p, st);
+    return cb_attn_launch_tensor(ctx, p, st);
 }

@@ -1,5 +1,13 @@
-// Tree attention: work decomposition shared by the tensor-core kernel, the CUDA-core kernel and the
-// split-KV combine pass.
+// Tree attention: work decomposition shared by the tensor-core kernel and the merge pass.
+//
+// Work is measured in key tiles of 128 keys.  Sequence b has tiles_b = ceil(ctx_b / 128) + 1 of them (the
+// last one holds the tree's own keys).  A unit is one (sequence, kv head, row group): a row group is a
+// pair of 128-row tiles (row = node_local * G + g, NPT = 128 / G nodes per tile), or a single tile when
+// the whole tree fits one tile; only row tiles that hold valid nodes form units.  All units, in
+// (sequence, kv head, row group) order, laid end to end give one global sequence of key tiles; it is cut
+// into `nc` equal ranges, one per persistent CTA (a stream-K split).  A CTA therefore finishes whole
+// units, plus at most one unit it shares with earlier CTAs and one it shares with later CTAs; shared
+// units leave unnormalised partials that the merge pass combines.
 #pragma once
 #include "cb_common.cuh"
 
@@ -18,23 +26,107 @@ struct CbAttnParams {
     const int32_t* n_nodes;
     __nv_bfloat16* out;
     float* lse;
-    float* part;          // [slot][128][D + 4]: unnormalised O row, running max (log2 domain), sum, 2 pad (rows stay 16-byte aligned)
+    float* part;          // [2 * nc slots][2 row tiles][128 rows][D + 4]: unnormalised O row, running max (log2 domain), sum
     int B, T, W, Hq, Hkv, G, D, P, max_pages, num_pages;
-    int NPT;              // tree nodes per row tile = 128 / G; a tile holds rows node_local * G + g
-    int MT;               // row tiles per (sequence, kv head) = ceil(T / NPT)
-    int nsplit;           // key splits per unit; 1 = write the output directly
+    int NPT;              // tree nodes per row tile = 128 / G
+    int MT;               // row tiles that T nodes need = ceil(T / NPT)
+    int nc;               // persistent CTAs (= ranges of the global tile sequence)
     float scale_log2;     // softmax scale * log2(e)
     uint32_t* status;
 };
 
-// Key tiles of sequence b: ceil(ctx / 128) context tiles followed by one tile holding the tree keys.
-// Split s of nsplit covers tiles [lo, hi).
-__device__ __forceinline__ void cb_split_range(int ctx, int nsplit, int s, int* lo, int* hi) {
-    const int tiles = (ctx + CB_KT - 1) / CB_KT + 1;
-    *lo = (int)(((long long)tiles * s) / nsplit);
-    *hi = (int)(((long long)tiles * (s + 1)) / nsplit);
+// Per-sequence shape of the decomposition.
+struct CbSeqShape {
+    int n, ctx, tiles, mtn, RG;
+    long long W;          // key tiles of all units of this sequence
+};
+
+__device__ __forceinline__ CbSeqShape cb_seq_shape(const CbAttnParams& p, int b) {
+    CbSeqShape s;
+    s.n = min(max(p.n_nodes[b], 0), p.T);
+    s.ctx = min(max(p.ctx_len[b], 0), p.max_pages * p.P);
+    s.tiles = (s.ctx + CB_KT - 1) / CB_KT + 1;
+    s.mtn = (s.n + p.NPT - 1) / p.NPT;
+    s.RG = p.MT == 1 ? (s.mtn > 0 ? 1 : 0) : (s.mtn + 1) / 2;
+    s.W = (long long)p.Hkv * s.RG * s.tiles;
+    return s;
 }
+
+__device__ __forceinline__ long long cb_range_start(long long total, int nc, int c) { return total * c / nc; }
+// CTA whose range holds global tile x.
+__device__ __forceinline__ int cb_cta_of(long long total, int nc, long long x) { return (int)(((x + 1) * nc - 1) / total); }
+
+// Warp-collective: total weight of all sequences, and the sequence holding global tile g (with the
+// global index at which that sequence starts).  Every lane gets the results.
+__device__ __forceinline__ long long cb_sched_total(const CbAttnParams& p, int lane) {
+    long long tot = 0;
+    for (int base = 0; base < p.B; base += 32) {
+        const int b = base + lane;
+        long long w = b < p.B ? cb_seq_shape(p, b).W : 0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) w += __shfl_xor_sync(CB_FULL, w, o);
+        tot += w;
+    }
+    return tot;
+}
+__device__ __forceinline__ void cb_sched_locate(const CbAttnParams& p, long long g, int lane, int* b_out, long long* pre_out) {
+    long long run = 0;
+    int fb = p.B;
+    long long fpre = 0;
+    for (int base = 0; base < p.B; base += 32) {
+        const int b = base + lane;
+        const long long w = b < p.B ? cb_seq_shape(p, b).W : 0;
+        long long inc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long t = __shfl_up_sync(CB_FULL, inc, o);
+            if (lane >= o) inc += t;
+        }
+        const long long pre = run + inc - w;
+        const uint32_t hit = __ballot_sync(CB_FULL, w > 0 && g >= pre && g < pre + w);
+        if (hit) {
+            const int l = __ffs(hit) - 1;
+            fb = base + l;
+            fpre = __shfl_sync(CB_FULL, pre, l);
+            break;
+        }
+        run += __shfl_sync(CB_FULL, inc, 31);
+    }
+    *b_out = fb;
+    *pre_out = fpre;
+}
+
+// One unit's share of a CTA's range.
+struct CbUnit {
+    int b, kh, rg, t0, t1, tiles, n, ctx, nrt;   // nrt = valid row tiles in the group (1 or 2)
+};
+
+// Walks the units of the range [g, g1).  Every role of a CTA runs its own copy and sees the same units.
+struct CbWalker {
+    long long g, g1, pre;
+    int b;
+    CbSeqShape s;
+    __device__ __forceinline__ void init(const CbAttnParams& p, long long g0, long long g1_, int b0, long long pre0) {
+        g = g0; g1 = g1_; b = b0; pre = pre0;
+        if (g < g1) s = cb_seq_shape(p, b);
+    }
+    __device__ __forceinline__ bool next(const CbAttnParams& p, CbUnit* u) {
+        if (g >= g1) return false;
+        while (g >= pre + s.W) { pre += s.W; ++b; s = cb_seq_shape(p, b); }
+        const long long off = g - pre;
+        const int j = (int)(off / s.tiles);
+        u->t0 = (int)(off - (long long)j * s.tiles);
+        const long long room = g1 - g;
+        u->t1 = (int)min((long long)s.tiles, (long long)u->t0 + room);
+        u->b = b; u->kh = j / s.RG; u->rg = j % s.RG; u->tiles = s.tiles; u->n = s.n; u->ctx = s.ctx;
+        u->nrt = p.MT == 1 ? 1 : min(2, s.mtn - 2 * u->rg);
+        g += u->t1 - u->t0;
+        return true;
+    }
+};
+
+#define CB_ATTN_MAX_CTAS 160   // upper bound on persistent CTAs (>= SM count); sizes the partial buffer
+static_assert(CB_ATTN_MAX_UNITS == 4 * CB_ATTN_MAX_CTAS, "partial buffer: two shared units of two row tiles per CTA");
 
 cb_status cb_attn_launch_cuda_cores(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t st);
 cb_status cb_attn_launch_tensor(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t st);
-cb_status cb_attn_launch_combine(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t st);

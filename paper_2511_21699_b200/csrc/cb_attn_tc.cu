@@ -1,16 +1,22 @@
 // Tree-masked attention on the 5th-generation tensor cores (tcgen05) with TMA-staged paged K/V.
 //
-// One CTA handles one (key split, row tile, sequence, kv head).  A row tile packs the GQA group times a
-// range of tree nodes into the 128 rows of one MMA tile: row r = node_local * G + g.  Key tiles hold 128
-// keys: ceil(ctx/128) tiles of cached keys (eight 16-token pages each, fetched page by page with TMA
-// through the block table) followed by one tile with the tree's own keys, masked by the ancestor bits.
+// Persistent kernel: one CTA per SM, each working through an equal share of the global sequence of key
+// tiles (see cb_attn.cuh).  A CTA holds up to two 128-row query tiles of a unit and streams that unit's
+// 128-key tiles through a ring of 128B-swizzled shared-memory slots (K and V tiles alternate in the
+// ring; eight 16-token pages per tile, fetched page by page with TMA through the block table).
 //
-// Warp roles (192 threads):
-//   warp 0      TMA producer: K and V tiles into a ring of 128B-swizzled shared-memory stages
-//   warp 1      MMA issuer (one lane): S = Q K^T into a double-buffered TMEM tile, then O += P V with
-//               P read from TMEM; owns the TMEM allocation
-//   warps 2..5  softmax: one thread per row; S from TMEM to registers, fp32 online softmax in the
-//               log2 domain with lazy rescaling of O, P written back to TMEM as packed bf16 over S
+// Warp roles (384 threads, three warpgroups):
+//   warp 0        TMA producer for K/V: runs ahead across unit boundaries, limited only by the ring
+//   warp 1        MMA issuer (one lane): S = Q K^T into TMEM, then O += P V with P read from TMEM;
+//                 owns the TMEM allocation (S0, S1, O0, O1: 4 x 128 columns)
+//   warp 2        TMA loader for the query tiles of each unit
+//   warp 3        writes the zero rows of padding nodes (node >= n_nodes)
+//   warps 4..7    softmax warpgroup 0, warps 8..11 softmax warpgroup 1: one thread per query row; S from
+//                 TMEM to registers, fp32 online softmax in the log2 domain with lazy rescaling of O,
+//                 P written back to TMEM as packed bf16 over S; epilogue of the unit
+// A unit with two valid row tiles gives one to each softmax warpgroup (both consume every key tile, so
+// the tensor pipe works on one tile's MMAs while the other tile is in softmax).  A unit with one valid
+// row tile is handled by warpgroup 0 alone with S double-buffered over S0/S1.
 // All waits are bounded; a wait that runs out records CB_ERR_TIMEOUT and the CTA drains and exits.
 #include <cuda.h>
 
@@ -18,11 +24,12 @@
 
 namespace {
 
-constexpr uint32_t kWaitLimit = 1u << 24;
-constexpr int kThreads = 192;
+constexpr long long kWaitCycles = 1ll << 32;     // bound of every wait, in SM clock cycles (about two seconds)
+constexpr uint32_t kSuspendNs = 20000;
+constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
 
-struct TcMaps { CUtensorMap k_pool, v_pool, k_tree, v_tree; };
+struct TcMaps { CUtensorMap k_pool, v_pool, k_tree, v_tree, q; };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -35,23 +42,26 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+// Potentially blocking test of a barrier phase: the hardware suspends the thread until the phase completes
+// or a time limit of about kSuspendNs passes, so waiting warps do not take issue slots from working ones.
+__device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
     return ok;
 }
-// Bounded wait. Returns false when the wait ran out or another role already gave up.
+// Bounded wait. Returns false when the wait ran out or another role already gave up; the first to run out
+// records CB_ERR_TIMEOUT and raises the CTA's abort flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
-    for (uint32_t it = 0; it < kWaitLimit; ++it) {
-        if (mbar_test(bar, parity)) return true;
-        if (it > 64) {
-            __nanosleep(40);
-            if ((it & 255u) == 0u && *abort_flag) return false;
-        }
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        if (mbar_try(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) break;
     }
     *abort_flag = 1;
     atomicCAS(status, 0u, (uint32_t)CB_ERR_TIMEOUT);
@@ -133,20 +143,30 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool b_mn_major)
            ((uint32_t)(M >> 4) << 24);
 }
 
+template <int REGS> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS)); }
+template <int REGS> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS)); }
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
 template <int D>
 struct Cfg {
     static constexpr int DB = D / 64;                        // 64-element (128-byte) column blocks per row
-    static constexpr int NST = (D == 128) ? 3 : 4;           // K/V stages
+    static constexpr int NSLOT = (D == 128) ? 5 : 8;         // ring slots, each one K or one V tile
     static constexpr uint32_t TILE_BYTES = CB_KT * D * 2;    // one K or V tile
-    static constexpr uint32_t Q_BYTES = CB_MT * D * 2;
-    static constexpr uint32_t OFF_Q = 0;
-    static constexpr uint32_t OFF_K = Q_BYTES;
-    static constexpr uint32_t OFF_V = OFF_K + NST * TILE_BYTES;
-    static constexpr uint32_t OFF_BAR = OFF_V + NST * TILE_BYTES;
-    static constexpr int NBAR = 1 + 3 * NST + 2 + 2 + 1;     // q, k_full, v_full, kv_free, s_full[2], p_ready[2], o_done
-    static constexpr uint32_t SMEM = OFF_BAR + NBAR * 8 + 16;
+    static constexpr uint32_t Q_BYTES = CB_MT * D * 2;       // one query row tile
+    static constexpr uint32_t OFF_Q = 0;                     // two row tiles
+    static constexpr uint32_t OFF_RING = 2 * Q_BYTES;
+    static constexpr uint32_t OFF_BAR = OFF_RING + NSLOT * TILE_BYTES;
+    // slot_full[NSLOT], slot_free[NSLOT], q_full, q_free, s_full[2], p_ready[2], o_free[2], pv_done[2][2]
+    static constexpr int NBAR = 2 * NSLOT + 2 + 10;
+    static constexpr uint32_t OFF_MISC = OFF_BAR + NBAR * 8;  // schedule, tmem base, abort flag
+    static constexpr uint32_t SMEM = OFF_MISC + 64;
     static constexpr uint32_t SMEM_ALLOC = SMEM + 1024;      // slack to align the base to 1024 bytes
+    static constexpr uint32_t O_COL = 256;                   // TMEM columns: S0 at 0, S1 at 128, O0 at 256, O1 at 256 + D
 };
+
+struct SchedSmem { long long g0, g1, pre0; int b0; };
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -156,272 +176,402 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* sgen = smem_raw + (sbase - smem_u32(smem_raw));
     const uint32_t bar0 = sbase + C::OFF_BAR;
-    const uint32_t bar_q = bar0;
-    auto bar_kfull = [&](int s) { return bar0 + 8u * (1 + s); };
-    auto bar_vfull = [&](int s) { return bar0 + 8u * (1 + C::NST + s); };
-    auto bar_free = [&](int s) { return bar0 + 8u * (1 + 2 * C::NST + s); };
-    auto bar_sfull = [&](int s) { return bar0 + 8u * (1 + 3 * C::NST + s); };
-    auto bar_pready = [&](int s) { return bar0 + 8u * (3 + 3 * C::NST + s); };
-    const uint32_t bar_odone = bar0 + 8u * (5 + 3 * C::NST);
-    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sgen + C::OFF_BAR + C::NBAR * 8);
-    volatile int* s_abort = reinterpret_cast<volatile int*>(sgen + C::OFF_BAR + C::NBAR * 8 + 4);
+    auto bar_full = [&](int s) { return bar0 + 8u * s; };
+    auto bar_free = [&](int s) { return bar0 + 8u * (C::NSLOT + s); };
+    const uint32_t bar_qfull = bar0 + 8u * (2 * C::NSLOT), bar_qfree = bar_qfull + 8u;
+    auto bar_sfull = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 2 + s); };
+    auto bar_pready = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 4 + s); };
+    auto bar_ofree = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 6 + s); };
+    // The k-th PV on accumulator `ol` completes on barrier (ol, k & 1) as that barrier's phase k >> 1.  Two
+    // alternating barriers keep a waiter that skips phases at most one phase behind (a parity wait needs that).
+    auto bar_pvdone = [&](int ol, uint32_t k) { return bar0 + 8u * (2 * C::NSLOT + 8 + ol * 2 + (k & 1u)); };
+    SchedSmem* s_sched = reinterpret_cast<SchedSmem*>(sgen + C::OFF_MISC);
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sgen + C::OFF_MISC + 32);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(sgen + C::OFF_MISC + 36);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int split = blockIdx.x, mt = blockIdx.y, bk = blockIdx.z;
-    const int b = bk / p.Hkv, kh = bk % p.Hkv;
-    const int n = p.n_nodes[b], ctx = p.ctx_len[b];
-    const int nct = (ctx + CB_KT - 1) / CB_KT;               // context tiles; tile nct is the tree tile
-    int t_lo, t_hi;
-    cb_split_range(ctx, p.nsplit, split, &t_lo, &t_hi);
-    const int ntiles = t_hi - t_lo;
-    const int RT = p.NPT * p.G;                               // rows of this tile that exist
+    const int cta = blockIdx.x;
+    const int RT = p.NPT * p.G;                               // rows of a row tile that exist
 
-    // Softmax-thread row bookkeeping (also used by the trivial path)
-    const int wq = warp & 3;
-    const int row = wq * 32 + lane;
-    const int node = mt * p.NPT + row / p.G, g = row % p.G, h = kh * p.G + g;
-    const bool row_exists = warp >= 2 && row < RT && node < p.T;
-    const bool row_valid = row_exists && node < n;
-    const size_t slot = ((size_t)bk * p.MT + mt) * p.nsplit + split;
-
-    if (n <= 0 || ntiles <= 0 || mt * p.NPT >= n) {
-        // Nothing to attend from this CTA: zero rows / an empty partial.
-        if (warp >= 2) {
-            if (p.nsplit == 1) {
-                if (row_exists) {
-                    uint4* op = reinterpret_cast<uint4*>(p.out + (((size_t)b * p.T + node) * p.Hq + h) * D);
-                    for (int c = 0; c < D / 8; ++c) op[c] = make_uint4(0, 0, 0, 0);
-                    if (p.lse) p.lse[((size_t)b * p.Hq + h) * p.T + node] = 0.f;
-                }
-            } else {
-                float* pp = p.part + (slot * CB_MT + row) * (D + 4);
-                pp[D] = -INFINITY; pp[D + 1] = 0.f;
-            }
-        }
-        return;
-    }
-
-    if (tid == 0) {
-        mbar_init(bar_q, 128);
-        for (int s = 0; s < C::NST; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_vfull(s), 1); mbar_init(bar_free(s), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(bar_sfull(s), 1); mbar_init(bar_pready(s), 128); }
-        mbar_init(bar_odone, 1);
-        *s_abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 1) {
+    if (warp == 0) {
+        // this CTA's range of the global tile sequence
+        const long long tot = cb_sched_total(p, lane);
+        const long long g0 = cb_range_start(tot, p.nc, cta), g1 = cb_range_start(tot, p.nc, cta + 1);
+        int b0 = 0;
+        long long pre0 = 0;
+        if (g0 < g1) cb_sched_locate(p, g0, lane, &b0, &pre0);
+        if (lane == 0) { s_sched->g0 = g0; s_sched->g1 = g1; s_sched->b0 = b0; s_sched->pre0 = pre0; }
+    } else if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else if (warp == 2) {
+        if (lane == 0) {
+            for (int s = 0; s < C::NSLOT; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_free(s), 1); }
+            mbar_init(bar_qfull, 1); mbar_init(bar_qfree, 1);
+            for (int s = 0; s < 2; ++s) {
+                mbar_init(bar_sfull(s), 1); mbar_init(bar_pready(s), 128); mbar_init(bar_ofree(s), 128);
+                mbar_init(bar_pvdone(s, 0), 1); mbar_init(bar_pvdone(s, 1), 1);
+            }
+            *s_abort = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            tma_prefetch_desc(&maps.k_pool); tma_prefetch_desc(&maps.v_pool); tma_prefetch_desc(&maps.q);
+            tma_prefetch_desc(&maps.k_tree); tma_prefetch_desc(&maps.v_tree);
+        }
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *s_tmem;
-    const uint32_t tm_S0 = tmem, tm_O = tmem + 256;           // S buffers at columns 0 and 128, O at 256
+    const long long g0 = s_sched->g0, g1 = s_sched->g1, pre0 = s_sched->pre0;
+    const int b0 = s_sched->b0;
+    CbWalker wk;
+    wk.init(p, g0, g1, b0, pre0);
+    CbUnit u;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        constexpr int NB = 8 * C::DB;                        // boxes (16 keys x 64 dims) per K tile
-        const bool active = lane < 2 * NB;
-        const bool isV = lane >= NB;
-        const int within = lane % NB, j = within % 8, dblk = within / 8;
-        const int npages = (ctx + p.P - 1) / p.P;
-        for (int it = 0; it < ntiles; ++it) {
-            const int tile = t_lo + it, st = it % C::NST;
-            if (it >= C::NST) {
-                if (!mbar_wait(bar_free(st), ((it / C::NST) - 1) & 1, s_abort, p.status)) break;
-            }
-            if (lane == 0) { mbar_expect_tx(bar_kfull(st), C::TILE_BYTES); mbar_expect_tx(bar_vfull(st), C::TILE_BYTES); }
-            __syncwarp();
-            if (active) {
-                const uint32_t dst = sbase + (isV ? C::OFF_V : C::OFF_K) + st * C::TILE_BYTES + dblk * (CB_KT * 128) + j * 2048;
-                const uint32_t bar = isV ? bar_vfull(st) : bar_kfull(st);
-                if (tile < nct) {
-                    const int pidx = tile * (CB_KT / 16) + j;
-                    // pages past the sequence's end are fetched out of range: the copy fills zeros
-                    const int page = pidx < npages ? p.block_table[(size_t)b * p.max_pages + pidx] : p.num_pages;
-                    tma_load_4d(dst, isV ? &maps.v_pool : &maps.k_pool, bar, dblk * 64, kh, 0, page);
-                } else {
-                    tma_load_4d(dst, isV ? &maps.v_tree : &maps.k_tree, bar, dblk * 64, kh, 16 * j, b);
+    if (warp < 4) {
+        reg_dealloc<120>();
+        if (warp == 0) {
+            // ------------------------------------------------------------------ K/V producer
+            constexpr int NB = 8 * C::DB;                    // boxes (16 keys x 64 dims) per tile
+            const bool active = lane < 2 * NB;
+            const bool isV = lane >= NB;
+            const int within = lane % NB, j = within % 8, dblk = within / 8;
+            uint32_t seq = 0;
+            bool ok = true;
+            while (ok && wk.next(p, &u)) {
+                const int npages = (u.ctx + p.P - 1) / p.P, nct = u.tiles - 1;
+                const int32_t* bt = p.block_table + (size_t)u.b * p.max_pages;
+                for (int i = u.t0; i < u.t1; ++i) {
+                    int page = p.num_pages;                  // out of range: the copy fills zeros
+                    if (active && i < nct) {
+                        const int pidx = i * (CB_KT / 16) + j;
+                        if (pidx < npages) page = bt[pidx];
+                    }
+                    const uint32_t ks = seq % C::NSLOT, vs = (seq + 1) % C::NSLOT;
+                    if (seq >= (uint32_t)C::NSLOT && !(ok = mbar_wait(bar_free(ks), (seq / C::NSLOT - 1) & 1, s_abort, p.status))) break;
+                    if (seq + 1 >= (uint32_t)C::NSLOT && !(ok = mbar_wait(bar_free(vs), ((seq + 1) / C::NSLOT - 1) & 1, s_abort, p.status))) break;
+                    if (lane == 0) { mbar_expect_tx(bar_full(ks), C::TILE_BYTES); mbar_expect_tx(bar_full(vs), C::TILE_BYTES); }
+                    __syncwarp();
+                    if (active) {
+                        const uint32_t sl = isV ? vs : ks;
+                        const uint32_t dst = sbase + C::OFF_RING + sl * C::TILE_BYTES + dblk * (CB_KT * 128) + j * 2048;
+                        if (i < nct) tma_load_4d(dst, isV ? &maps.v_pool : &maps.k_pool, bar_full(sl), dblk * 64, u.kh, 0, page);
+                        else tma_load_4d(dst, isV ? &maps.v_tree : &maps.k_tree, bar_full(sl), dblk * 64, u.kh, 16 * j, u.b);
+                    }
+                    seq += 2;
                 }
             }
-        }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = make_idesc(128, CB_KT, false);
-            constexpr uint32_t idesc_o = make_idesc(128, D, true);
-            bool ok = mbar_wait(bar_q, 0, s_abort, p.status);
-            tc_fence_after();
-            for (int it = 0; ok && it <= ntiles; ++it) {
-                if (it < ntiles) {
-                    const int st = it % C::NST, sb = it & 1;
-                    if (!(ok = mbar_wait(bar_kfull(st), (it / C::NST) & 1, s_abort, p.status))) break;
-                    tc_fence_after();
-                    const uint32_t qa = sbase + C::OFF_Q, ka = sbase + C::OFF_K + st * C::TILE_BYTES;
+        } else if (warp == 1) {
+            // ------------------------------------------------------------------ MMA issuer
+            if (lane == 0) {
+                constexpr uint32_t idesc_s = make_idesc(128, CB_KT, false);
+                constexpr uint32_t idesc_o = make_idesc(128, D, true);
+                uint32_t seq = 0, uq = 0, c_p[2] = {0u, 0u}, c_of[2] = {0u, 0u}, c_pv[2] = {0u, 0u};
+                bool ok = true;
+                auto issue_s = [&](int rt, int buf, uint32_t kslot) {
+                    const uint32_t qa = sbase + C::OFF_Q + rt * C::Q_BYTES, ka = sbase + C::OFF_RING + kslot * C::TILE_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
                         const uint32_t off = (kk / 4) * (CB_KT * 128) + (kk % 4) * 32;
-                        mma_ss(tm_S0 + sb * 128, make_desc(qa + off, 16, 1024), make_desc(ka + off, 16, 1024), idesc_s, kk > 0);
+                        mma_ss(tmem + buf * 128, make_desc(qa + off, 16, 1024), make_desc(ka + off, 16, 1024), idesc_s, kk > 0);
                     }
-                    tc_commit(bar_sfull(sb));
-                }
-                if (it >= 1) {
-                    const int pt = it - 1, st = pt % C::NST, sb = pt & 1;
-                    if (!(ok = mbar_wait(bar_vfull(st), (pt / C::NST) & 1, s_abort, p.status))) break;
-                    if (!(ok = mbar_wait(bar_pready(sb), (pt >> 1) & 1, s_abort, p.status))) break;
-                    tc_fence_after();
-                    const uint32_t va = sbase + C::OFF_V + st * C::TILE_BYTES;
+                };
+                auto issue_pv = [&](int ol, int buf, uint32_t vslot, bool accum) {
+                    const uint32_t va = sbase + C::OFF_RING + vslot * C::TILE_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < CB_KT / 16; ++kk)
-                        mma_ts(tm_O, tm_S0 + sb * 128 + kk * 8, make_desc(va + kk * 2048, CB_KT * 128, 1024), idesc_o,
-                               (pt > 0 || kk > 0) ? 1u : 0u);
-                    tc_commit(bar_free(st));
-                    tc_commit(bar_odone);
+                        mma_ts(tmem + C::O_COL + ol * D, tmem + buf * 128 + kk * 8, make_desc(va + kk * 2048, CB_KT * 128, 1024), idesc_o,
+                               (accum || kk > 0) ? 1u : 0u);
+                };
+                while (ok && wk.next(p, &u)) {
+                    const bool two = u.nrt == 2;
+                    if (!(ok = mbar_wait(bar_qfull, uq & 1, s_abort, p.status))) break;
+                    tc_fence_after();
+                    const uint32_t seq0 = seq;
+                    for (int i = u.t0; ok && i <= u.t1; ++i) {
+                        const uint32_t kseq = seq0 + 2 * (i - u.t0), vseq_prev = kseq - 1;
+                        const uint32_t ks = kseq % C::NSLOT, vs = vseq_prev % C::NSLOT;
+                        if (two) {
+                            // per row tile l: PV of the previous key tile, then S of this one, so that the other
+                            // tile's softmax always has MMAs to overlap with
+                            for (int l = 0; l < 2; ++l) {
+                                if (i > u.t0) {
+                                    if (l == 0 && !(ok = mbar_wait(bar_full(vs), (vseq_prev / C::NSLOT) & 1, s_abort, p.status))) break;
+                                    if (!(ok = mbar_wait(bar_pready(l), c_p[l] & 1, s_abort, p.status))) break;
+                                    ++c_p[l];
+                                    if (i == u.t0 + 1) {
+                                        if (c_of[l] > 0 && !(ok = mbar_wait(bar_ofree(l), (c_of[l] - 1) & 1, s_abort, p.status))) break;
+                                        ++c_of[l];
+                                    }
+                                    tc_fence_after();
+                                    issue_pv(l, l, vs, i > u.t0 + 1);
+                                    tc_commit(bar_pvdone(l, c_pv[l]));
+                                    ++c_pv[l];
+                                    if (l == 1) tc_commit(bar_free(vs));
+                                }
+                                if (i < u.t1) {
+                                    if (l == 0) {
+                                        if (!(ok = mbar_wait(bar_full(ks), (kseq / C::NSLOT) & 1, s_abort, p.status))) break;
+                                        tc_fence_after();
+                                    }
+                                    issue_s(l, l, ks);
+                                    tc_commit(bar_sfull(l));
+                                    if (l == 1) {
+                                        tc_commit(bar_free(ks));
+                                        if (i == u.t1 - 1) tc_commit(bar_qfree);
+                                    }
+                                }
+                            }
+                        } else {
+                            if (i < u.t1) {
+                                const int buf = (i - u.t0) & 1;
+                                if (!(ok = mbar_wait(bar_full(ks), (kseq / C::NSLOT) & 1, s_abort, p.status))) break;
+                                tc_fence_after();
+                                issue_s(0, buf, ks);
+                                tc_commit(bar_sfull(buf));
+                                tc_commit(bar_free(ks));
+                                if (i == u.t1 - 1) tc_commit(bar_qfree);
+                            }
+                            if (i > u.t0) {
+                                const int buf = (i - 1 - u.t0) & 1;
+                                if (!(ok = mbar_wait(bar_full(vs), (vseq_prev / C::NSLOT) & 1, s_abort, p.status))) break;
+                                if (!(ok = mbar_wait(bar_pready(buf), c_p[buf] & 1, s_abort, p.status))) break;
+                                ++c_p[buf];
+                                if (i == u.t0 + 1) {
+                                    if (c_of[0] > 0 && !(ok = mbar_wait(bar_ofree(0), (c_of[0] - 1) & 1, s_abort, p.status))) break;
+                                    ++c_of[0];
+                                }
+                                tc_fence_after();
+                                issue_pv(0, buf, vs, i > u.t0 + 1);
+                                tc_commit(bar_pvdone(0, c_pv[0]));
+                                ++c_pv[0];
+                                tc_commit(bar_free(vs));
+                            }
+                        }
+                    }
+                    seq = seq0 + 2 * (u.t1 - u.t0);
+                    ++uq;
                 }
             }
+            __syncwarp();
+        } else if (warp == 2) {
+            // ------------------------------------------------------------------ query loader
+            if (lane == 0) {
+                uint32_t uq = 0;
+                while (wk.next(p, &u)) {
+                    if (uq > 0 && !mbar_wait(bar_qfree, (uq - 1) & 1, s_abort, p.status)) break;
+                    mbar_expect_tx(bar_qfull, (uint32_t)(u.nrt * C::DB * RT * 128));
+                    for (int rt = 0; rt < u.nrt; ++rt)
+                        for (int db = 0; db < C::DB; ++db)
+                            tma_load_4d(sbase + C::OFF_Q + rt * C::Q_BYTES + db * (CB_MT * 128), &maps.q, bar_qfull, db * 64, u.kh * p.G,
+                                        (u.rg * 2 + rt) * p.NPT, u.b);
+                    ++uq;
+                }
+            }
+            __syncwarp();
+        } else {
+            // ------------------------------------------------------------------ zero rows of padding nodes
+            const int per_row = p.Hq * D / 8;                // 16-byte chunks per node row
+            for (int idx = cta; idx < p.B * p.T; idx += gridDim.x) {
+                const int b = idx / p.T, node = idx % p.T;
+                const int n = min(max(p.n_nodes[b], 0), p.T);
+                if (node < n) continue;
+                uint4* op = reinterpret_cast<uint4*>(p.out + (size_t)idx * p.Hq * D);
+                for (int k = lane; k < per_row; k += 32) op[k] = make_uint4(0, 0, 0, 0);
+                if (p.lse) for (int h = lane; h < p.Hq; h += 32) p.lse[((size_t)b * p.Hq + h) * p.T + node] = 0.f;
+            }
         }
-        __syncwarp();
     } else {
-        // ------------------------------------------------------------------ softmax / correction / epilogue
-        // Q tile -> shared memory in the 128B-swizzled K-major layout: row r, 16-byte chunk c of column
-        // block db lands at db * 16 KB + r * 128 + ((c ^ (r & 7)) * 16).
-        {
-            constexpr int CPR = C::DB * 8, RPI = 32 / CPR;          // 16-byte chunks per row, rows per iteration
-            const int sub = lane / CPR, cc = lane % CPR, db = cc / 8, ch = cc % 8;
-            for (int k = 0; k < 32 / RPI; ++k) {
-                const int r = wq * 32 + k * RPI + sub;
-                const int nd = mt * p.NPT + r / p.G, hh = kh * p.G + r % p.G;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (r < RT && nd < n)
-                    v = *reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.T + nd) * p.Hq + hh) * D + db * 64 + ch * 8);
-                *reinterpret_cast<uint4*>(sgen + C::OFF_Q + db * (CB_MT * 128) + r * 128 + ((ch ^ (r & 7)) << 4)) = v;
-            }
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(bar_q);
-
-        uint32_t mrow[4] = {0u, 0u, 0u, 0u};
-        if (row_valid) for (int k = 0; k < p.W; ++k) mrow[k] = p.tree_mask[((size_t)b * p.T + node) * p.W + k];
-        float m_used = -INFINITY, l = 0.f;
+        // ---------------------------------------------------------------------- softmax / correction / epilogue
+        reg_alloc<192>();
+        const int wg = (warp - 4) >> 2;                       // softmax warpgroup = row tile of a two-tile unit
+        const int wq = warp & 3;                              // TMEM lane quarter this warp may access
+        const int row = wq * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+        const uint32_t tm_O = tmem + C::O_COL + wg * D + lane_addr;
+        uint32_t c_s[2] = {0u, 0u};                           // completions of s_full[k] so far (consumed by either warpgroup)
+        uint32_t c_pv = 0;                                    // PV completions on this warpgroup's O so far
         bool ok = true;
-        for (int it = 0; it < ntiles; ++it) {
-            const int tile = t_lo + it, sb = it & 1;
-            if (!(ok = mbar_wait(bar_sfull(sb), (it >> 1) & 1, s_abort, p.status))) break;
-            tc_fence_after();
-            uint32_t sr[128];
-            const uint32_t ts = tm_S0 + sb * 128 + lane_addr;
-            CB_TMEM_LD32(sr, 0, ts);
-            CB_TMEM_LD32(sr, 32, ts + 32);
-            CB_TMEM_LD32(sr, 64, ts + 64);
-            CB_TMEM_LD32(sr, 96, ts + 96);
-            tmem_wait_ld();
-            const bool is_tree = tile == nct;
-            const int kv = is_tree ? n : min(CB_KT, ctx - tile * CB_KT);
-            float mloc = -INFINITY;
-            if (!row_valid) {
-#pragma unroll
-                for (int jx = 0; jx < 128; ++jx) sr[jx] = 0xFF800000u;
-            } else if (is_tree) {
-#pragma unroll
-                for (int jx = 0; jx < 128; ++jx) {
-                    const bool vis = (mrow[jx >> 5] >> (jx & 31)) & 1u;
-                    if (!vis || jx >= kv) sr[jx] = 0xFF800000u;
-                    mloc = fmaxf(mloc, __uint_as_float(sr[jx]));
+        while (ok && wk.next(p, &u)) {
+            const bool two = u.nrt == 2;
+            const int nt = u.t1 - u.t0;
+            if (wg == 1 && !two) {
+                // Handled by warpgroup 0 alone.  This warpgroup still observes every S completion, in order: a
+                // parity wait is only meaningful for a waiter that is at most one phase away from the barrier.
+                for (int i = u.t0; ok && i < u.t1; ++i) {
+                    const int buf = (i - u.t0) & 1;
+                    ok = mbar_wait(bar_sfull(buf), c_s[buf] & 1, s_abort, p.status);
+                    ++c_s[buf];
                 }
-            } else if (kv < CB_KT) {
-#pragma unroll
-                for (int jx = 0; jx < 128; ++jx) {
-                    if (jx >= kv) sr[jx] = 0xFF800000u;
-                    mloc = fmaxf(mloc, __uint_as_float(sr[jx]));
-                }
-            } else {
-#pragma unroll
-                for (int jx = 0; jx < 128; ++jx) mloc = fmaxf(mloc, __uint_as_float(sr[jx]));
+                continue;
             }
-            mloc *= p.scale_log2;
-            // lazy rescaling: keep the reference maximum until the running maximum exceeds it by 2^8
-            const bool need = mloc > m_used + 8.0f;
-            const float alpha = need ? ex2(m_used - mloc) : 1.0f;
-            if (need) m_used = mloc;
-            if (it > 0) {
-                if (!(ok = mbar_wait(bar_odone, (it - 1) & 1, s_abort, p.status))) break;
-                tc_fence_after();
-                if (__any_sync(CB_FULL, need)) {
+            const int rt = u.rg * 2 + wg;
+            const int node = rt * p.NPT + row / p.G, g = row % p.G, h = u.kh * p.G + g;
+            const bool row_valid = row < RT && node < u.n;
+            const bool warp_active = (wq * 32) < RT && (rt * p.NPT + (wq * 32) / p.G) < u.n;   // row 0 of the warp is valid
+            const int nct = u.tiles - 1;
+            uint32_t mrow[4] = {0u, 0u, 0u, 0u};
+            if (row_valid) {
+                const uint32_t* mp = p.tree_mask + ((size_t)u.b * p.T + node) * p.W;
+                mrow[0] = mp[0];
+                if (p.W > 1) mrow[1] = mp[1];
+                if (p.W > 2) mrow[2] = mp[2];
+                if (p.W > 3) mrow[3] = mp[3];
+            }
+            float m_used = -INFINITY, l = 0.f;
+            for (int i = u.t0; i < u.t1; ++i) {
+                const int buf = two ? wg : ((i - u.t0) & 1);
+                if (!(ok = mbar_wait(bar_sfull(buf), c_s[buf] & 1, s_abort, p.status))) break;
+                ++c_s[buf];
+                if (i - u.t0 >= 2) {
+                    // PV(i-2) finished before S(i) was issued; observing it keeps this waiter in step with the barrier
+                    const uint32_t k = c_pv + (uint32_t)(i - u.t0) - 2u;
+                    if (!(ok = mbar_wait(bar_pvdone(wg, k), (k >> 1) & 1, s_abort, p.status))) break;
+                }
+                if (warp_active) {
+                    tc_fence_after();
+                    const uint32_t ts = tmem + buf * 128 + lane_addr;
+                    // visibility of the tile's 128 keys for this row: context keys below ctx, tree keys by the ancestor bits
+                    const bool is_tree = i == nct;
+                    const int kv = is_tree ? u.n : min(CB_KT, u.ctx - i * CB_KT);
+                    uint32_t vm[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int lo = kv - 32 * k;
+                        const uint32_t below = lo >= 32 ? 0xFFFFFFFFu : (lo <= 0 ? 0u : ((1u << lo) - 1u));
+                        vm[k] = row_valid ? (is_tree ? (mrow[k] & below) : below) : 0u;
+                    }
+                    const bool all_vis = __all_sync(CB_FULL, (vm[0] & vm[1] & vm[2] & vm[3]) == 0xFFFFFFFFu);
+                    // pass 1: row maximum of the visible scores
+                    float mloc = -INFINITY;
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t sr[64];
+                        CB_TMEM_LD32(sr, 0, ts + half * 64);
+                        CB_TMEM_LD32(sr, 32, ts + half * 64 + 32);
+                        tmem_wait_ld();
+                        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+                        if (all_vis) {
+#pragma unroll
+                            for (int jx = 0; jx < 64; jx += 4) {
+                                m0 = fmaxf(m0, __uint_as_float(sr[jx])); m1 = fmaxf(m1, __uint_as_float(sr[jx + 1]));
+                                m2 = fmaxf(m2, __uint_as_float(sr[jx + 2])); m3 = fmaxf(m3, __uint_as_float(sr[jx + 3]));
+                            }
+                        } else {
+#pragma unroll
+                            for (int jx = 0; jx < 64; ++jx) {
+                                const bool vis = (vm[half * 2 + (jx >> 5)] >> (jx & 31)) & 1u;
+                                m0 = fmaxf(m0, vis ? __uint_as_float(sr[jx]) : -INFINITY);
+                            }
+                        }
+                        mloc = fmaxf(mloc, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
+                    }
+                    mloc *= p.scale_log2;
+                    // lazy rescaling: keep the reference maximum until the running maximum exceeds it by 2^8
+                    const bool need = mloc > m_used + 8.0f;
+                    const float alpha = need ? ex2(m_used - mloc) : 1.0f;
+                    if (need) m_used = mloc;
+                    if (i > u.t0 && __any_sync(CB_FULL, need)) {
+                        // O must be complete up to the previous tile before it is rescaled
+                        const uint32_t k = c_pv + (uint32_t)(i - u.t0) - 1u;
+                        if (!(ok = mbar_wait(bar_pvdone(wg, k), (k >> 1) & 1, s_abort, p.status))) break;
+                        tc_fence_after();
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t o[32];
+                            CB_TMEM_LD32(o, 0, tm_O + c * 32);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int jx = 0; jx < 32; ++jx) o[jx] = __float_as_uint(__uint_as_float(o[jx]) * alpha);
+                            CB_TMEM_ST32(o, 0, tm_O + c * 32);
+                        }
+                    }
+                    l *= alpha;
+                    const float mu = (m_used == -INFINITY) ? 0.f : m_used;
+                    // pass 2: P = 2^(s * scale - m), written back over S as packed bf16 (64 scores -> 32 columns)
+                    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t sr[64];
+                        CB_TMEM_LD32(sr, 0, ts + half * 64);
+                        CB_TMEM_LD32(sr, 32, ts + half * 64 + 32);
+                        tmem_wait_ld();
+                        if (!all_vis) {
+#pragma unroll
+                            for (int jx = 0; jx < 64; ++jx)
+                                if (!((vm[half * 2 + (jx >> 5)] >> (jx & 31)) & 1u)) sr[jx] = 0xFF800000u;
+                        }
+                        uint32_t pk[32];
+#pragma unroll
+                        for (int jx = 0; jx < 64; jx += 4) {
+                            const float p0 = ex2(fmaf(__uint_as_float(sr[jx]), p.scale_log2, -mu));
+                            const float p1 = ex2(fmaf(__uint_as_float(sr[jx + 1]), p.scale_log2, -mu));
+                            const float p2 = ex2(fmaf(__uint_as_float(sr[jx + 2]), p.scale_log2, -mu));
+                            const float p3 = ex2(fmaf(__uint_as_float(sr[jx + 3]), p.scale_log2, -mu));
+                            l0 += p0; l1 += p1; l2 += p2; l3 += p3;
+                            pk[jx >> 1] = pack_bf16(p0, p1);
+                            pk[(jx >> 1) + 1] = pack_bf16(p2, p3);
+                        }
+                        CB_TMEM_ST32(pk, 0, ts + half * 32);
+                    }
+                    l += (l0 + l1) + (l2 + l3);
+                    tmem_wait_st();
+                }
+                tc_fence_before();
+                mbar_arrive(bar_pready(buf));
+            }
+            if (!ok) break;
+            // ---- epilogue of this unit's share: O is complete once its last PV has finished
+            {
+                const uint32_t k = c_pv + (uint32_t)nt - 1u;
+                if (!(ok = mbar_wait(bar_pvdone(wg, k), (k >> 1) & 1, s_abort, p.status))) break;
+            }
+            c_pv += (uint32_t)nt;
+            if (two) c_s[1 - wg] += (uint32_t)nt;            // the other warpgroup consumed those
+            tc_fence_after();
+            if (warp_active) {
+                const bool whole = u.t0 == 0 && u.t1 == u.tiles;
+                if (whole) {
+                    const float inv = l > 0.f ? 1.0f / l : 0.f;
 #pragma unroll
                     for (int c = 0; c < D / 32; ++c) {
                         uint32_t o[32];
-                        CB_TMEM_LD32(o, 0, tm_O + lane_addr + c * 32);
+                        CB_TMEM_LD32(o, 0, tm_O + c * 32);
                         tmem_wait_ld();
+                        if (row_valid) {
+                            uint4* op = reinterpret_cast<uint4*>(p.out + (((size_t)u.b * p.T + node) * p.Hq + h) * D + c * 32);
 #pragma unroll
-                        for (int jx = 0; jx < 32; ++jx) o[jx] = __float_as_uint(__uint_as_float(o[jx]) * alpha);
-                        CB_TMEM_ST32(o, 0, tm_O + lane_addr + c * 32);
-                    }
-                }
-            }
-            l *= alpha;
-            const float mu = (m_used == -INFINITY) ? 0.f : m_used;
-            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-            uint32_t pk[64];
-#pragma unroll
-            for (int jx = 0; jx < 128; jx += 4) {
-                const float p0 = ex2(fmaf(__uint_as_float(sr[jx]), p.scale_log2, -mu));
-                const float p1 = ex2(fmaf(__uint_as_float(sr[jx + 1]), p.scale_log2, -mu));
-                const float p2 = ex2(fmaf(__uint_as_float(sr[jx + 2]), p.scale_log2, -mu));
-                const float p3 = ex2(fmaf(__uint_as_float(sr[jx + 3]), p.scale_log2, -mu));
-                l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                pk[jx >> 1] = pack_bf16(p0, p1);
-                pk[(jx >> 1) + 1] = pack_bf16(p2, p3);
-            }
-            l += (l0 + l1) + (l2 + l3);
-            CB_TMEM_ST32(pk, 0, ts);
-            CB_TMEM_ST32(pk, 32, ts + 32);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar_pready(sb));
-        }
-        if (ok) ok = mbar_wait(bar_odone, (ntiles - 1) & 1, s_abort, p.status);
-        tc_fence_after();
-        if (ok) {
-            if (p.nsplit == 1) {
-                const float inv = (row_valid && l > 0.f) ? 1.0f / l : 0.f;
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    CB_TMEM_LD32(o, 0, tm_O + lane_addr + c * 32);
-                    tmem_wait_ld();
-                    if (row_exists) {
-                        uint4* op = reinterpret_cast<uint4*>(p.out + (((size_t)b * p.T + node) * p.Hq + h) * D + c * 32);
-#pragma unroll
-                        for (int v4 = 0; v4 < 4; ++v4) {
-                            uint4 w;
-                            w.x = pack_bf16(__uint_as_float(o[v4 * 8 + 0]) * inv, __uint_as_float(o[v4 * 8 + 1]) * inv);
-                            w.y = pack_bf16(__uint_as_float(o[v4 * 8 + 2]) * inv, __uint_as_float(o[v4 * 8 + 3]) * inv);
-                            w.z = pack_bf16(__uint_as_float(o[v4 * 8 + 4]) * inv, __uint_as_float(o[v4 * 8 + 5]) * inv);
-                            w.w = pack_bf16(__uint_as_float(o[v4 * 8 + 6]) * inv, __uint_as_float(o[v4 * 8 + 7]) * inv);
-                            op[v4] = w;
+                            for (int v4 = 0; v4 < 4; ++v4) {
+                                uint4 w;
+                                w.x = pack_bf16(__uint_as_float(o[v4 * 8 + 0]) * inv, __uint_as_float(o[v4 * 8 + 1]) * inv);
+                                w.y = pack_bf16(__uint_as_float(o[v4 * 8 + 2]) * inv, __uint_as_float(o[v4 * 8 + 3]) * inv);
+                                w.z = pack_bf16(__uint_as_float(o[v4 * 8 + 4]) * inv, __uint_as_float(o[v4 * 8 + 5]) * inv);
+                                w.w = pack_bf16(__uint_as_float(o[v4 * 8 + 6]) * inv, __uint_as_float(o[v4 * 8 + 7]) * inv);
+                                op[v4] = w;
+                            }
                         }
                     }
-                }
-                if (row_exists && p.lse)
-                    p.lse[((size_t)b * p.Hq + h) * p.T + node] = (row_valid && l > 0.f) ? (m_used + log2f(l)) * 0.6931471805599453f : 0.f;
-            } else {
-                float* pp = p.part + (slot * CB_MT + row) * (D + 4);
+                    if (row_valid && p.lse)
+                        p.lse[((size_t)u.b * p.Hq + h) * p.T + node] = l > 0.f ? (m_used + log2f(l)) * 0.6931471805599453f : 0.f;
+                } else {
+                    const size_t slot = 2 * (size_t)cta + (u.t0 == 0 ? 1 : 0);
+                    float* pp = p.part + ((slot * 2 + wg) * CB_MT + row) * (D + 4);
 #pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    CB_TMEM_LD32(o, 0, tm_O + lane_addr + c * 32);
-                    tmem_wait_ld();
-                    if (row_valid) {
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        CB_TMEM_LD32(o, 0, tm_O + c * 32);
+                        tmem_wait_ld();
+                        if (row_valid) {
 #pragma unroll
-                        for (int v4 = 0; v4 < 8; ++v4)
-                            *reinterpret_cast<uint4*>(pp + c * 32 + v4 * 4) = make_uint4(o[v4 * 4], o[v4 * 4 + 1], o[v4 * 4 + 2], o[v4 * 4 + 3]);
+                            for (int v4 = 0; v4 < 8; ++v4)
+                                *reinterpret_cast<uint4*>(pp + c * 32 + v4 * 4) = make_uint4(o[v4 * 4], o[v4 * 4 + 1], o[v4 * 4 + 2], o[v4 * 4 + 3]);
+                        }
                     }
+                    if (row_valid) { pp[D] = m_used; pp[D + 1] = l; }
                 }
-                pp[D] = row_valid ? m_used : -INFINITY;
-                pp[D + 1] = row_valid ? l : 0.f;
             }
+            tc_fence_before();
+            mbar_arrive(bar_ofree(wg));
         }
     }
 
@@ -435,6 +585,63 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// Merge pass: block (c, *) looks at the unit that CTA c of the attention kernel started but did not finish,
+// and combines the partials that CTA c and the following CTAs left for it.  One warp per output row.
+template <int D>
+__global__ void __launch_bounds__(256) cb_attn_merge_kernel(const CbAttnParams p) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c = blockIdx.x;
+    const long long tot = cb_sched_total(p, lane);
+    if (tot <= 0) return;
+    const long long g0 = cb_range_start(tot, p.nc, c), g1 = cb_range_start(tot, p.nc, c + 1);
+    if (g1 <= g0 || g1 >= tot) return;                        // empty range, or the last range
+    int b;
+    long long pre;
+    cb_sched_locate(p, g1 - 1, lane, &b, &pre);
+    const CbSeqShape s = cb_seq_shape(p, b);
+    const long long off = g1 - 1 - pre;
+    const int j = (int)(off / s.tiles);
+    if ((int)(off - (long long)j * s.tiles) == s.tiles - 1) return;   // the unit ends with this range
+    const long long ustart = pre + (long long)j * s.tiles;
+    if (ustart < g0) return;                                  // started by an earlier CTA: that CTA's block merges it
+    const int c_last = cb_cta_of(tot, p.nc, ustart + s.tiles - 1);
+    const int kh = j / s.RG, rg = j % s.RG;
+    const int nrt = p.MT == 1 ? 1 : min(2, s.mtn - 2 * rg);
+    const int RT = p.NPT * p.G;
+    constexpr int PER = D / 32;
+    const size_t rstride = (size_t)(D + 4), sstride = (size_t)2 * CB_MT * rstride;
+    for (int r2 = blockIdx.y * 8 + warp; r2 < nrt * CB_MT; r2 += gridDim.y * 8) {
+        const int wg = r2 / CB_MT, row = r2 % CB_MT;
+        const int node = (rg * 2 + wg) * p.NPT + row / p.G, h = kh * p.G + row % p.G;
+        if (row >= RT || node >= s.n) continue;
+        float M = -INFINITY;
+        for (int cc = c; cc <= c_last; ++cc) {
+            if (cb_range_start(tot, p.nc, cc) == cb_range_start(tot, p.nc, cc + 1)) continue;
+            const size_t slot = 2 * (size_t)cc + (cc == c ? 1 : 0);
+            M = fmaxf(M, p.part[slot * sstride + ((size_t)wg * CB_MT + row) * rstride + D]);
+        }
+        float o[PER], Lsum = 0.f;
+#pragma unroll
+        for (int d = 0; d < PER; ++d) o[d] = 0.f;
+        for (int cc = c; cc <= c_last; ++cc) {
+            if (cb_range_start(tot, p.nc, cc) == cb_range_start(tot, p.nc, cc + 1)) continue;
+            const size_t slot = 2 * (size_t)cc + (cc == c ? 1 : 0);
+            const float* pp = p.part + slot * sstride + ((size_t)wg * CB_MT + row) * rstride;
+            const float ms = pp[D];
+            if (ms == -INFINITY) continue;
+            const float w = exp2f(ms - M);
+            Lsum += w * pp[D + 1];
+#pragma unroll
+            for (int d = 0; d < PER; ++d) o[d] = fmaf(w, pp[lane * PER + d], o[d]);
+        }
+        const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
+        __nv_bfloat16* op = p.out + (((size_t)b * p.T + node) * p.Hq + h) * D + lane * PER;
+#pragma unroll
+        for (int d = 0; d < PER; ++d) op[d] = __float2bfloat16_rn(o[d] * inv);
+        if (p.lse && lane == 0) p.lse[((size_t)b * p.Hq + h) * p.T + node] = Lsum > 0.f ? (M + log2f(Lsum)) * 0.6931471805599453f : 0.f;
     }
 }
 
@@ -454,19 +661,19 @@ EncodeTiledFn get_encode() {
     return fn;
 }
 
-// 4-D view (d, kv head, row, block) of a [blocks, rows, Hkv, D] bf16 tensor; box = 64 dims x 1 head x 16 rows.
-bool encode_kv_map(CUtensorMap* m, const void* base, int D, int Hkv, int rows, long blocks) {
+// 4-D view (d, head, row, block) of a [blocks, rows, heads, D] bf16 tensor; box = 64 dims x box_heads x box_rows.
+bool encode_map(CUtensorMap* m, const void* base, int D, int heads, int rows, long blocks, int box_heads, int box_rows) {
     EncodeTiledFn enc = get_encode();
     if (!enc) { fprintf(stderr, "cacheback: cuTensorMapEncodeTiled entry point not found\n"); return false; }
-    cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)Hkv, (cuuint64_t)rows, (cuuint64_t)blocks};
-    cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)Hkv * D * 2, (cuuint64_t)rows * Hkv * D * 2};
-    cuuint32_t box[4] = {64, 1, 16, 1};
+    cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)heads, (cuuint64_t)rows, (cuuint64_t)blocks};
+    cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)heads * D * 2, (cuuint64_t)rows * heads * D * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
-        fprintf(stderr, "cacheback: tensor map encode failed (%d): D=%d Hkv=%d rows=%d blocks=%ld base=%p\n", (int)r, D, Hkv, rows,
+        fprintf(stderr, "cacheback: tensor map encode failed (%d): D=%d heads=%d rows=%d blocks=%ld base=%p\n", (int)r, D, heads, rows,
                 blocks, base);
     return r == CUDA_SUCCESS;
 }
@@ -478,9 +685,10 @@ cb_status launch(const CbAttnParams& p, const TcMaps& maps, cudaStream_t st) {
         CB_CUDA(cudaFuncSetAttribute(cb_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<D>::SMEM_ALLOC));
         attr_set = true;
     }
-    dim3 grid(p.nsplit, p.MT, p.B * p.Hkv);
-    cb_attn_tc_kernel<D><<<grid, kThreads, Cfg<D>::SMEM_ALLOC, st>>>(p, maps);
-    cb_count_launch(1);
+    cb_attn_tc_kernel<D><<<p.nc, kThreads, Cfg<D>::SMEM_ALLOC, st>>>(p, maps);
+    CB_CUDA(cudaGetLastError());
+    cb_attn_merge_kernel<D><<<dim3(p.nc, 4), 256, 0, st>>>(p);
+    cb_count_launch(2);
     CB_CUDA(cudaGetLastError());
     return CB_OK;
 }
@@ -491,9 +699,10 @@ cb_status cb_attn_launch_tensor(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t
     (void)ctx;
     if (p.P != 16) return CB_ERR_UNSUPPORTED;
     TcMaps maps;
-    if (!encode_kv_map(&maps.k_pool, p.k_pool, p.D, p.Hkv, p.P, p.num_pages)) return CB_ERR_CUDA;
-    if (!encode_kv_map(&maps.v_pool, p.v_pool, p.D, p.Hkv, p.P, p.num_pages)) return CB_ERR_CUDA;
-    if (!encode_kv_map(&maps.k_tree, p.k_tree, p.D, p.Hkv, p.T, p.B)) return CB_ERR_CUDA;
-    if (!encode_kv_map(&maps.v_tree, p.v_tree, p.D, p.Hkv, p.T, p.B)) return CB_ERR_CUDA;
+    if (!encode_map(&maps.k_pool, p.k_pool, p.D, p.Hkv, p.P, p.num_pages, 1, 16)) return CB_ERR_CUDA;
+    if (!encode_map(&maps.v_pool, p.v_pool, p.D, p.Hkv, p.P, p.num_pages, 1, 16)) return CB_ERR_CUDA;
+    if (!encode_map(&maps.k_tree, p.k_tree, p.D, p.Hkv, p.T, p.B, 1, 16)) return CB_ERR_CUDA;
+    if (!encode_map(&maps.v_tree, p.v_tree, p.D, p.Hkv, p.T, p.B, 1, 16)) return CB_ERR_CUDA;
+    if (!encode_map(&maps.q, p.q, p.D, p.Hq, p.T, p.B, p.G, p.NPT)) return CB_ERR_CUDA;
     return p.D == 128 ? launch<128>(p, maps, st) : launch<64>(p, maps, st);
 }

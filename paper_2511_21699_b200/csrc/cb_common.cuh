@@ -73,9 +73,9 @@ struct cb_ctx {
     unsigned long long* d_counters;  // [CB_NUM_COUNTERS]
     unsigned long long* d_rowmax;    // [batch * max_nodes] packed (value, index) maxima, zero between calls
     uint32_t* d_ticket;     // [batch] CTAs-finished counters, zero between calls
-    float* d_attn_part;     // split-KV partial outputs
+    float* d_attn_part;     // partial outputs of units shared between CTAs
     size_t attn_part_floats;
-    int attn_max_units;     // partial slots available
+    int attn_max_units;     // partial row tiles available
     int num_sms;
 };
 
@@ -89,7 +89,7 @@ struct CbLayout {
 cb_status cb_compute_layout(const cb_config* cfg, CbLayout* L);
 void cb_count_launch(int n);
 
-#define CB_ATTN_MAX_UNITS 1024  // split-KV partial slots (each 128 rows x (D + 4) floats)
+#define CB_ATTN_MAX_UNITS 640   // partial row tiles (128 rows x (D + 4) floats): 2 shared units x 2 row tiles per persistent CTA, 160 CTAs
 
 #define CB_CHECK_ARG(cond) do { if (!(cond)) return CB_ERR_INVALID_ARG; } while (0)
 #include <stdio.h>
