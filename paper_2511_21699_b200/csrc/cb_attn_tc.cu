@@ -441,7 +441,8 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                         const uint32_t below = lo >= 32 ? 0xFFFFFFFFu : (lo <= 0 ? 0u : ((1u << lo) - 1u));
                         vm[k] = row_valid ? (is_tree ? (mrow[k] & below) : below) : 0u;
                     }
-                    const bool all_vis = __all_sync(CB_FULL, (vm[0] & vm[1] & vm[2] & vm[3]) == 0xFFFFFFFFu);
+                    // rows that do not exist take the fast path too: whatever they compute stays in their own row
+                    const bool all_vis = __all_sync(CB_FULL, !row_valid || (vm[0] & vm[1] & vm[2] & vm[3]) == 0xFFFFFFFFu);
                     // pass 1: row maximum of the visible scores
                     float mloc = -INFINITY;
 #pragma unroll
