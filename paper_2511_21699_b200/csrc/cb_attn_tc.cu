@@ -114,6 +114,12 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
     asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, " \
                  "%12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, "   \
                  "%31};" ::CB_W32(a, o), "r"(taddr) : "memory")
+#define CB_RW32(a) "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]), "+r"(a[8]), \
+    "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]), "+r"(a[16]), "+r"(a[17]), "+r"(a[18]), \
+    "+r"(a[19]), "+r"(a[20]), "+r"(a[21]), "+r"(a[22]), "+r"(a[23]), "+r"(a[24]), "+r"(a[25]), "+r"(a[26]), "+r"(a[27]), "+r"(a[28]), \
+    "+r"(a[29]), "+r"(a[30]), "+r"(a[31])
+// Waits for this thread's outstanding TMEM loads; naming the destination registers keeps their uses below the wait.
+#define CB_TMEM_WAIT_LD32(a) asm volatile("tcgen05.wait::ld.sync.aligned;" : CB_RW32(a) :: "memory")
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -121,6 +127,23 @@ __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+// Two fp32 values in one 64-bit register pair, for the packed fp32x2 arithmetic of sm_100.
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     uint32_t r;
@@ -141,6 +164,52 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
            ((uint32_t)(M >> 4) << 24);
+}
+
+// Low and high 32-bit words of a shared-memory matrix descriptor (128-byte swizzle, 1024-byte stride between
+// 8-row groups).  All operands live below 256 KB, so stepping the low word by (bytes >> 4) moves the start address.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) { return ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16); }
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+
+// One MMA issuer thread feeds the tensor pipe, so the instructions between two MMAs are kept to a minimum: each
+// of the blocks below issues all MMAs of one 128 x 128 x D (or 128 x D x 128) product from a single asm statement.
+#define CB_MMA_SS_STEP(OFF)                                                                                          \
+    "add.u32 ra, %1, " #OFF ";\n\tadd.u32 rb, %2, " #OFF ";\n\tmov.b64 da, {ra, %3};\n\tmov.b64 db, {rb, %3};\n\t"  \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
+// S[tmem] = Q[smem, K-major] * K[smem, K-major]^T over D.  qlo / klo: low descriptor words of the first 16-wide slice.
+template <int D>
+__device__ __forceinline__ void mma_s_block(uint32_t d_tmem, uint32_t qlo, uint32_t klo, uint32_t idesc) {
+    if (D == 128) {
+        asm volatile(
+            "{\n\t.reg .pred pt, pf;\n\t.reg .b64 da, db;\n\t.reg .b32 ra, rb;\n\t"
+            "setp.eq.u32 pt, %4, %4;\n\tsetp.ne.u32 pf, %4, %4;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pf;\n\t"
+            CB_MMA_SS_STEP(2) CB_MMA_SS_STEP(4) CB_MMA_SS_STEP(6) CB_MMA_SS_STEP(1024) CB_MMA_SS_STEP(1026) CB_MMA_SS_STEP(1028)
+            CB_MMA_SS_STEP(1030) "}"
+            ::"r"(d_tmem), "r"(qlo), "r"(klo), "r"(kDescHi), "r"(idesc) : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred pt, pf;\n\t.reg .b64 da, db;\n\t.reg .b32 ra, rb;\n\t"
+            "setp.eq.u32 pt, %4, %4;\n\tsetp.ne.u32 pf, %4, %4;\n\t"
+            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pf;\n\t"
+            CB_MMA_SS_STEP(2) CB_MMA_SS_STEP(4) CB_MMA_SS_STEP(6) "}"
+            ::"r"(d_tmem), "r"(qlo), "r"(klo), "r"(kDescHi), "r"(idesc) : "memory");
+    }
+}
+#define CB_MMA_TS_STEP(K)                                                                                            \
+    "add.u32 ra, %1, 8 * " #K ";\n\tadd.u32 rb, %2, 128 * " #K ";\n\tmov.b64 db, {rb, %3};\n\t"                     \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], [ra], db, %4, pt;\n\t"
+// O[tmem] (+)= P[tmem, packed bf16] * V[smem, MN-major] over the tile's 128 keys.  vlo: low descriptor word of the V tile.
+__device__ __forceinline__ void mma_pv_block(uint32_t d_tmem, uint32_t p_tmem, uint32_t vlo, uint32_t idesc, uint32_t accum) {
+    asm volatile(
+        "{\n\t.reg .pred pt, pa;\n\t.reg .b64 db;\n\t.reg .b32 ra, rb;\n\t"
+        "setp.eq.u32 pt, %4, %4;\n\tsetp.ne.u32 pa, %5, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, pa;\n\t"
+        CB_MMA_TS_STEP(1) CB_MMA_TS_STEP(2) CB_MMA_TS_STEP(3) CB_MMA_TS_STEP(4) CB_MMA_TS_STEP(5) CB_MMA_TS_STEP(6) CB_MMA_TS_STEP(7) "}"
+        ::"r"(d_tmem), "r"(p_tmem), "r"(vlo), "r"(kDescHi), "r"(idesc), "r"(accum) : "memory");
 }
 
 template <int REGS> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS)); }
@@ -268,20 +337,13 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                 constexpr uint32_t idesc_o = make_idesc(128, D, true);
                 uint32_t seq = 0, uq = 0, c_p[2] = {0u, 0u}, c_of[2] = {0u, 0u}, c_pv[2] = {0u, 0u};
                 bool ok = true;
+                const uint32_t q_lo0 = desc_lo(sbase + C::OFF_Q, 16), k_lo0 = desc_lo(sbase + C::OFF_RING, 16);
+                const uint32_t v_lo0 = desc_lo(sbase + C::OFF_RING, CB_KT * 128);
                 auto issue_s = [&](int rt, int buf, uint32_t kslot) {
-                    const uint32_t qa = sbase + C::OFF_Q + rt * C::Q_BYTES, ka = sbase + C::OFF_RING + kslot * C::TILE_BYTES;
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = (kk / 4) * (CB_KT * 128) + (kk % 4) * 32;
-                        mma_ss(tmem + buf * 128, make_desc(qa + off, 16, 1024), make_desc(ka + off, 16, 1024), idesc_s, kk > 0);
-                    }
+                    mma_s_block<D>(tmem + buf * 128, q_lo0 + rt * (C::Q_BYTES >> 4), k_lo0 + kslot * (C::TILE_BYTES >> 4), idesc_s);
                 };
                 auto issue_pv = [&](int ol, int buf, uint32_t vslot, bool accum) {
-                    const uint32_t va = sbase + C::OFF_RING + vslot * C::TILE_BYTES;
-#pragma unroll
-                    for (int kk = 0; kk < CB_KT / 16; ++kk)
-                        mma_ts(tmem + C::O_COL + ol * D, tmem + buf * 128 + kk * 8, make_desc(va + kk * 2048, CB_KT * 128, 1024), idesc_o,
-                               (accum || kk > 0) ? 1u : 0u);
+                    mma_pv_block(tmem + C::O_COL + ol * D, tmem + buf * 128, v_lo0 + vslot * (C::TILE_BYTES >> 4), idesc_o, accum ? 1u : 0u);
                 };
                 while (ok && wk.next(p, &u)) {
                     const bool two = u.nrt == 2;
@@ -443,30 +505,29 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     }
                     // rows that do not exist take the fast path too: whatever they compute stays in their own row
                     const bool all_vis = __all_sync(CB_FULL, !row_valid || (vm[0] & vm[1] & vm[2] & vm[3]) == 0xFFFFFFFFu);
-                    // pass 1: row maximum of the visible scores
-                    float mloc = -INFINITY;
+                    // pass 1: row maximum of the visible scores, 32 columns at a time with the next 32 in flight
+                    uint32_t sa[32], sb[32];
+                    CB_TMEM_LD32(sa, 0, ts);
+                    float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t sr[64];
-                        CB_TMEM_LD32(sr, 0, ts + half * 64);
-                        CB_TMEM_LD32(sr, 32, ts + half * 64 + 32);
-                        tmem_wait_ld();
-                        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t* cur = (c & 1) ? sb : sa;
+                        uint32_t* nxt = (c & 1) ? sa : sb;
+                        CB_TMEM_WAIT_LD32(cur);
+                        if (c < 3) CB_TMEM_LD32(nxt, 0, ts + 32 * (c + 1));
                         if (all_vis) {
 #pragma unroll
-                            for (int jx = 0; jx < 64; jx += 4) {
-                                m0 = fmaxf(m0, __uint_as_float(sr[jx])); m1 = fmaxf(m1, __uint_as_float(sr[jx + 1]));
-                                m2 = fmaxf(m2, __uint_as_float(sr[jx + 2])); m3 = fmaxf(m3, __uint_as_float(sr[jx + 3]));
+                            for (int jx = 0; jx < 32; jx += 4) {
+                                m0 = fmaxf(m0, __uint_as_float(cur[jx])); m1 = fmaxf(m1, __uint_as_float(cur[jx + 1]));
+                                m2 = fmaxf(m2, __uint_as_float(cur[jx + 2])); m3 = fmaxf(m3, __uint_as_float(cur[jx + 3]));
                             }
                         } else {
 #pragma unroll
-                            for (int jx = 0; jx < 64; ++jx) {
-                                const bool vis = (vm[half * 2 + (jx >> 5)] >> (jx & 31)) & 1u;
-                                m0 = fmaxf(m0, vis ? __uint_as_float(sr[jx]) : -INFINITY);
-                            }
+                            for (int jx = 0; jx < 32; ++jx) m0 = fmaxf(m0, ((vm[c] >> jx) & 1u) ? __uint_as_float(cur[jx]) : -INFINITY);
                         }
-                        mloc = fmaxf(mloc, fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)));
                     }
+                    float mloc = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+                    CB_TMEM_LD32(sa, 0, ts);                     // first columns of pass 2, in flight during the bookkeeping below
                     mloc *= p.scale_log2;
                     // lazy rescaling: keep the reference maximum until the running maximum exceeds it by 2^8
                     const bool need = mloc > m_used + 8.0f;
@@ -490,31 +551,36 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     l *= alpha;
                     const float mu = (m_used == -INFINITY) ? 0.f : m_used;
                     // pass 2: P = 2^(s * scale - m), written back over S as packed bf16 (64 scores -> 32 columns)
-                    float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+                    const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), negmu2 = f2_pack(-mu, -mu);
+                    uint64_t lsa = f2_pack(0.f, 0.f), lsb = f2_pack(0.f, 0.f);
+                    uint32_t pk[32];
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t sr[64];
-                        CB_TMEM_LD32(sr, 0, ts + half * 64);
-                        CB_TMEM_LD32(sr, 32, ts + half * 64 + 32);
-                        tmem_wait_ld();
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t* cur = (c & 1) ? sb : sa;
+                        uint32_t* nxt = (c & 1) ? sa : sb;
+                        CB_TMEM_WAIT_LD32(cur);
+                        if (c < 3) CB_TMEM_LD32(nxt, 0, ts + 32 * (c + 1));
                         if (!all_vis) {
 #pragma unroll
-                            for (int jx = 0; jx < 64; ++jx)
-                                if (!((vm[half * 2 + (jx >> 5)] >> (jx & 31)) & 1u)) sr[jx] = 0xFF800000u;
+                            for (int jx = 0; jx < 32; ++jx)
+                                if (!((vm[c] >> jx) & 1u)) cur[jx] = 0xFF800000u;
                         }
-                        uint32_t pk[32];
 #pragma unroll
-                        for (int jx = 0; jx < 64; jx += 4) {
-                            const float p0 = ex2(fmaf(__uint_as_float(sr[jx]), p.scale_log2, -mu));
-                            const float p1 = ex2(fmaf(__uint_as_float(sr[jx + 1]), p.scale_log2, -mu));
-                            const float p2 = ex2(fmaf(__uint_as_float(sr[jx + 2]), p.scale_log2, -mu));
-                            const float p3 = ex2(fmaf(__uint_as_float(sr[jx + 3]), p.scale_log2, -mu));
-                            l0 += p0; l1 += p1; l2 += p2; l3 += p3;
-                            pk[jx >> 1] = pack_bf16(p0, p1);
-                            pk[(jx >> 1) + 1] = pack_bf16(p2, p3);
+                        for (int jx = 0; jx < 32; jx += 4) {
+                            float p0, p1, p2, p3;
+                            f2_unpack(f2_fma(f2_pack(__uint_as_float(cur[jx]), __uint_as_float(cur[jx + 1])), scale2, negmu2), p0, p1);
+                            f2_unpack(f2_fma(f2_pack(__uint_as_float(cur[jx + 2]), __uint_as_float(cur[jx + 3])), scale2, negmu2), p2, p3);
+                            p0 = ex2(p0); p1 = ex2(p1); p2 = ex2(p2); p3 = ex2(p3);
+                            lsa = f2_add(lsa, f2_pack(p0, p1));
+                            lsb = f2_add(lsb, f2_pack(p2, p3));
+                            pk[(c & 1) * 16 + (jx >> 1)] = pack_bf16(p0, p1);
+                            pk[(c & 1) * 16 + (jx >> 1) + 1] = pack_bf16(p2, p3);
                         }
-                        CB_TMEM_ST32(pk, 0, ts + half * 32);
+                        if (c & 1) CB_TMEM_ST32(pk, 0, ts + (c >> 1) * 32);
                     }
+                    float l0, l1, l2, l3;
+                    f2_unpack(lsa, l0, l1);
+                    f2_unpack(lsb, l2, l3);
                     l += (l0 + l1) + (l2 + l3);
                     tmem_wait_st();
                 }
