@@ -20,6 +20,8 @@
 // All waits are bounded; a wait that runs out records CB_ERR_TIMEOUT and the CTA drains and exits.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "cb_attn.cuh"
 
 namespace {
@@ -79,21 +81,6 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accum) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accum) : "memory");
-}
-
 #define CB_R32(a, o) "=r"(a[o + 0]), "=r"(a[o + 1]), "=r"(a[o + 2]), "=r"(a[o + 3]), "=r"(a[o + 4]), "=r"(a[o + 5]), \
     "=r"(a[o + 6]), "=r"(a[o + 7]), "=r"(a[o + 8]), "=r"(a[o + 9]), "=r"(a[o + 10]), "=r"(a[o + 11]), "=r"(a[o + 12]), \
     "=r"(a[o + 13]), "=r"(a[o + 14]), "=r"(a[o + 15]), "=r"(a[o + 16]), "=r"(a[o + 17]), "=r"(a[o + 18]), "=r"(a[o + 19]), \
@@ -151,15 +138,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return r;
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle, for tiles whose rows are 128 bytes (64 bf16).
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)(lbo_bytes >> 4) << 16;
-    d |= (uint64_t)(sbo_bytes >> 4) << 32;
-    d |= 1ull << 46;
-    d |= 2ull << 61;
-    return d;
-}
 // Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major or MN-major.
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
@@ -227,8 +205,8 @@ struct Cfg {
     static constexpr uint32_t OFF_Q = 0;                     // two row tiles
     static constexpr uint32_t OFF_RING = 2 * Q_BYTES;
     static constexpr uint32_t OFF_BAR = OFF_RING + NSLOT * TILE_BYTES;
-    // slot_full[NSLOT], slot_free[NSLOT], q_full, q_free, s_full[2], p_ready[2], o_free[2], pv_done[2][2]
-    static constexpr int NBAR = 2 * NSLOT + 2 + 10;
+    // slot_full[NSLOT], slot_free[NSLOT], q_full, q_free, s_full0, p_ready[2], o_free[2]
+    static constexpr int NBAR = 2 * NSLOT + 2 + 5;
     static constexpr uint32_t OFF_MISC = OFF_BAR + NBAR * 8;  // schedule, tmem base, abort flag
     static constexpr uint32_t SMEM = OFF_MISC + 64;
     static constexpr uint32_t SMEM_ALLOC = SMEM + 1024;      // slack to align the base to 1024 bytes
@@ -248,12 +226,14 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     auto bar_full = [&](int s) { return bar0 + 8u * s; };
     auto bar_free = [&](int s) { return bar0 + 8u * (C::NSLOT + s); };
     const uint32_t bar_qfull = bar0 + 8u * (2 * C::NSLOT), bar_qfree = bar_qfull + 8u;
-    auto bar_sfull = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 2 + s); };
-    auto bar_pready = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 4 + s); };
-    auto bar_ofree = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 6 + s); };
-    // The k-th PV on accumulator `ol` completes on barrier (ol, k & 1) as that barrier's phase k >> 1.  Two
-    // alternating barriers keep a waiter that skips phases at most one phase behind (a parity wait needs that).
-    auto bar_pvdone = [&](int ol, uint32_t k) { return bar0 + 8u * (2 * C::NSLOT + 8 + ol * 2 + (k & 1u)); };
+    // Completion of the tensor core's work is signalled with as few commits as possible (a second commit behind the
+    // same MMA block stalls the issuer): a ring slot's "free" barrier doubles as "the S product that read this K tile is
+    // done" and "the PV product that read this V tile is done".  Its phases are a ring revolution apart, so a softmax
+    // thread can wait on it by the slot's sequence number alone.  Only row tile 0 of a two-row-tile unit needs a
+    // barrier of its own for S, because its S is finished before the K tile is released.
+    const uint32_t bar_sfull0 = bar0 + 8u * (2 * C::NSLOT + 2);
+    auto bar_pready = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 3 + s); };
+    auto bar_ofree = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 5 + s); };
     SchedSmem* s_sched = reinterpret_cast<SchedSmem*>(sgen + C::OFF_MISC);
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sgen + C::OFF_MISC + 32);
     volatile int* s_abort = reinterpret_cast<volatile int*>(sgen + C::OFF_MISC + 36);
@@ -276,10 +256,9 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     } else if (warp == 2) {
         if (lane == 0) {
             for (int s = 0; s < C::NSLOT; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_free(s), 1); }
-            mbar_init(bar_qfull, 1); mbar_init(bar_qfree, 1);
+            mbar_init(bar_qfull, 1); mbar_init(bar_qfree, 1); mbar_init(bar_sfull0, 1);
             for (int s = 0; s < 2; ++s) {
-                mbar_init(bar_sfull(s), 1); mbar_init(bar_pready(s), 128); mbar_init(bar_ofree(s), 128);
-                mbar_init(bar_pvdone(s, 0), 1); mbar_init(bar_pvdone(s, 1), 1);
+                mbar_init(bar_pready(s), 128); mbar_init(bar_ofree(s), 128);
             }
             *s_abort = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -335,7 +314,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             if (lane == 0) {
                 constexpr uint32_t idesc_s = make_idesc(128, CB_KT, false);
                 constexpr uint32_t idesc_o = make_idesc(128, D, true);
-                uint32_t seq = 0, uq = 0, c_p[2] = {0u, 0u}, c_of[2] = {0u, 0u}, c_pv[2] = {0u, 0u};
+                uint32_t seq = 0, uq = 0, c_p[2] = {0u, 0u}, c_of[2] = {0u, 0u};
                 bool ok = true;
                 const uint32_t q_lo0 = desc_lo(sbase + C::OFF_Q, 16), k_lo0 = desc_lo(sbase + C::OFF_RING, 16);
                 const uint32_t v_lo0 = desc_lo(sbase + C::OFF_RING, CB_KT * 128);
@@ -367,8 +346,6 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                                     }
                                     tc_fence_after();
                                     issue_pv(l, l, vs, i > u.t0 + 1);
-                                    tc_commit(bar_pvdone(l, c_pv[l]));
-                                    ++c_pv[l];
                                     if (l == 1) tc_commit(bar_free(vs));
                                 }
                                 if (i < u.t1) {
@@ -377,8 +354,9 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                                         tc_fence_after();
                                     }
                                     issue_s(l, l, ks);
-                                    tc_commit(bar_sfull(l));
-                                    if (l == 1) {
+                                    if (l == 0) {
+                                        tc_commit(bar_sfull0);
+                                    } else {
                                         tc_commit(bar_free(ks));
                                         if (i == u.t1 - 1) tc_commit(bar_qfree);
                                     }
@@ -390,7 +368,6 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                                 if (!(ok = mbar_wait(bar_full(ks), (kseq / C::NSLOT) & 1, s_abort, p.status))) break;
                                 tc_fence_after();
                                 issue_s(0, buf, ks);
-                                tc_commit(bar_sfull(buf));
                                 tc_commit(bar_free(ks));
                                 if (i == u.t1 - 1) tc_commit(bar_qfree);
                             }
@@ -405,8 +382,6 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                                 }
                                 tc_fence_after();
                                 issue_pv(0, buf, vs, i > u.t0 + 1);
-                                tc_commit(bar_pvdone(0, c_pv[0]));
-                                ++c_pv[0];
                                 tc_commit(bar_free(vs));
                             }
                         }
@@ -451,22 +426,30 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
         const int row = wq * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
         const uint32_t tm_O = tmem + C::O_COL + wg * D + lane_addr;
-        uint32_t c_s[2] = {0u, 0u};                           // completions of s_full[k] so far (consumed by either warpgroup)
-        uint32_t c_pv = 0;                                    // PV completions on this warpgroup's O so far
+        uint32_t c_s0 = 0;                                    // completions of s_full0 consumed so far (warpgroup 0 only)
+        uint32_t seq = 0;                                     // ring sequence number of the next unit's first K tile
         bool ok = true;
         while (ok && wk.next(p, &u)) {
             const bool two = u.nrt == 2;
             const int nt = u.t1 - u.t0;
+            const uint32_t seq0 = seq;
+            seq += 2u * (uint32_t)nt;
             if (wg == 1 && !two) {
-                // Handled by warpgroup 0 alone.  This warpgroup still observes every S completion, in order: a
-                // parity wait is only meaningful for a waiter that is at most one phase away from the barrier.
+                // Handled by warpgroup 0 alone.  This warpgroup still watches every S completion, in order: waiting on a
+                // barrier by parity is only sound for a thread that is at most one phase away from it, and a thread that
+                // ran ahead over this unit would later meet ring barriers that are whole revolutions behind it.
                 for (int i = u.t0; ok && i < u.t1; ++i) {
-                    const int buf = (i - u.t0) & 1;
-                    ok = mbar_wait(bar_sfull(buf), c_s[buf] & 1, s_abort, p.status);
-                    ++c_s[buf];
+                    const uint32_t kseq = seq0 + 2u * (uint32_t)(i - u.t0);
+                    ok = mbar_wait(bar_free(kseq % C::NSLOT), (kseq / C::NSLOT) & 1, s_abort, p.status);
                 }
                 continue;
             }
+            // S(i) is done when tile i's K slot is released (or, for row tile 0 of two, when s_full0 completes);
+            // every PV up to tile i is done when tile i's V slot is released.
+            auto wait_pv = [&](int i) {
+                const uint32_t vseq = seq0 + 2u * (uint32_t)(i - u.t0) + 1u;
+                return mbar_wait(bar_free(vseq % C::NSLOT), (vseq / C::NSLOT) & 1, s_abort, p.status);
+            };
             const int rt = u.rg * 2 + wg;
             const int node = rt * p.NPT + row / p.G, g = row % p.G, h = u.kh * p.G + g;
             const bool row_valid = row < RT && node < u.n;
@@ -483,12 +466,12 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             float m_used = -INFINITY, l = 0.f;
             for (int i = u.t0; i < u.t1; ++i) {
                 const int buf = two ? wg : ((i - u.t0) & 1);
-                if (!(ok = mbar_wait(bar_sfull(buf), c_s[buf] & 1, s_abort, p.status))) break;
-                ++c_s[buf];
-                if (i - u.t0 >= 2) {
-                    // PV(i-2) finished before S(i) was issued; observing it keeps this waiter in step with the barrier
-                    const uint32_t k = c_pv + (uint32_t)(i - u.t0) - 2u;
-                    if (!(ok = mbar_wait(bar_pvdone(wg, k), (k >> 1) & 1, s_abort, p.status))) break;
+                if (two && wg == 0) {
+                    if (!(ok = mbar_wait(bar_sfull0, c_s0 & 1, s_abort, p.status))) break;
+                    ++c_s0;
+                } else {
+                    const uint32_t kseq = seq0 + 2u * (uint32_t)(i - u.t0);
+                    if (!(ok = mbar_wait(bar_free(kseq % C::NSLOT), (kseq / C::NSLOT) & 1, s_abort, p.status))) break;
                 }
                 if (warp_active) {
                     tc_fence_after();
@@ -535,8 +518,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     if (need) m_used = mloc;
                     if (i > u.t0 && __any_sync(CB_FULL, need)) {
                         // O must be complete up to the previous tile before it is rescaled
-                        const uint32_t k = c_pv + (uint32_t)(i - u.t0) - 1u;
-                        if (!(ok = mbar_wait(bar_pvdone(wg, k), (k >> 1) & 1, s_abort, p.status))) break;
+                        if (!(ok = wait_pv(i - 1))) break;
                         tc_fence_after();
 #pragma unroll
                         for (int c = 0; c < D / 32; ++c) {
@@ -589,12 +571,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             }
             if (!ok) break;
             // ---- epilogue of this unit's share: O is complete once its last PV has finished
-            {
-                const uint32_t k = c_pv + (uint32_t)nt - 1u;
-                if (!(ok = mbar_wait(bar_pvdone(wg, k), (k >> 1) & 1, s_abort, p.status))) break;
-            }
-            c_pv += (uint32_t)nt;
-            if (two) c_s[1 - wg] += (uint32_t)nt;            // the other warpgroup consumed those
+            if (!(ok = wait_pv(u.t1 - 1))) break;
             tc_fence_after();
             if (warp_active) {
                 const bool whole = u.t0 == 0 && u.t1 == u.tiles;
@@ -679,30 +656,53 @@ __global__ void __launch_bounds__(256) cb_attn_merge_kernel(const CbAttnParams p
     const int nrt = p.MT == 1 ? 1 : min(2, s.mtn - 2 * rg);
     const int RT = p.NPT * p.G;
     constexpr int PER = D / 32;
+    // partial slots of this unit, listed once per block: CTA c's "started here" slot, then the "continued" slots of
+    // the following CTAs that have a non-empty range
+    __shared__ int s_slot[CB_ATTN_MAX_CTAS];
+    __shared__ int s_nparts;
+    if (warp == 0) {
+        int np = 0;
+        for (int base = c; base <= c_last; base += 32) {
+            const int cc = base + lane;
+            const bool valid = cc <= c_last && cb_range_start(tot, p.nc, cc) < cb_range_start(tot, p.nc, cc + 1);
+            const uint32_t m = __ballot_sync(CB_FULL, valid);
+            if (valid) s_slot[np + __popc(m & ((1u << lane) - 1u))] = 2 * cc + (cc == c ? 1 : 0);
+            np += __popc(m);
+        }
+        if (lane == 0) s_nparts = np;
+    }
+    __syncthreads();
+    const int nparts = s_nparts;
     const size_t rstride = (size_t)(D + 4), sstride = (size_t)2 * CB_MT * rstride;
     for (int r2 = blockIdx.y * 8 + warp; r2 < nrt * CB_MT; r2 += gridDim.y * 8) {
         const int wg = r2 / CB_MT, row = r2 % CB_MT;
         const int node = (rg * 2 + wg) * p.NPT + row / p.G, h = kh * p.G + row % p.G;
         if (row >= RT || node >= s.n) continue;
+        const float* base = p.part + ((size_t)wg * CB_MT + row) * rstride;
+        // lanes fetch the running maxima of up to 32 parts at a time
         float M = -INFINITY;
-        for (int cc = c; cc <= c_last; ++cc) {
-            if (cb_range_start(tot, p.nc, cc) == cb_range_start(tot, p.nc, cc + 1)) continue;
-            const size_t slot = 2 * (size_t)cc + (cc == c ? 1 : 0);
-            M = fmaxf(M, p.part[slot * sstride + ((size_t)wg * CB_MT + row) * rstride + D]);
+        for (int k0 = 0; k0 < nparts; k0 += 32) {
+            const int k = k0 + lane;
+            const float ms = k < nparts ? base[(size_t)s_slot[k] * sstride + D] : -INFINITY;
+            M = fmaxf(M, ms);
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(CB_FULL, M, o));
         float o[PER], Lsum = 0.f;
 #pragma unroll
         for (int d = 0; d < PER; ++d) o[d] = 0.f;
-        for (int cc = c; cc <= c_last; ++cc) {
-            if (cb_range_start(tot, p.nc, cc) == cb_range_start(tot, p.nc, cc + 1)) continue;
-            const size_t slot = 2 * (size_t)cc + (cc == c ? 1 : 0);
-            const float* pp = p.part + slot * sstride + ((size_t)wg * CB_MT + row) * rstride;
+        for (int k = 0; k < nparts; ++k) {
+            const float* pp = base + (size_t)s_slot[k] * sstride;
             const float ms = pp[D];
-            if (ms == -INFINITY) continue;
-            const float w = exp2f(ms - M);
-            Lsum += w * pp[D + 1];
-#pragma unroll
-            for (int d = 0; d < PER; ++d) o[d] = fmaf(w, pp[lane * PER + d], o[d]);
+            const float w = ms == -INFINITY ? 0.f : exp2f(ms - M);
+            Lsum = fmaf(w, pp[D + 1], Lsum);
+            if constexpr (PER == 4) {
+                const float4 v = *reinterpret_cast<const float4*>(pp + lane * 4);
+                o[0] = fmaf(w, v.x, o[0]); o[1] = fmaf(w, v.y, o[1]); o[2] = fmaf(w, v.z, o[2]); o[3] = fmaf(w, v.w, o[3]);
+            } else {
+                const float2 v = *reinterpret_cast<const float2*>(pp + lane * 2);
+                o[0] = fmaf(w, v.x, o[0]); o[1] = fmaf(w, v.y, o[1]);
+            }
         }
         const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
         __nv_bfloat16* op = p.out + (((size_t)b * p.T + node) * p.Hq + h) * D + lane * PER;
@@ -762,14 +762,45 @@ cb_status launch(const CbAttnParams& p, const TcMaps& maps, cudaStream_t st) {
 
 }  // namespace
 
+// Encoding five tensor maps costs several microseconds of host time, which matters at batch 1: the maps of the most
+// recent argument sets are kept (they depend only on the base pointers and the shape).
+namespace {
+struct MapKey {
+    const void *q, *k_pool, *v_pool, *k_tree, *v_tree;
+    int D, Hq, Hkv, P, T, B, G, NPT, num_pages;
+    bool operator==(const MapKey& o) const {
+        return q == o.q && k_pool == o.k_pool && v_pool == o.v_pool && k_tree == o.k_tree && v_tree == o.v_tree && D == o.D && Hq == o.Hq &&
+               Hkv == o.Hkv && P == o.P && T == o.T && B == o.B && G == o.G && NPT == o.NPT && num_pages == o.num_pages;
+    }
+};
+constexpr int kMapCache = 16;
+MapKey g_map_keys[kMapCache];
+TcMaps g_map_vals[kMapCache];
+int g_map_used = 0, g_map_next = 0;
+std::mutex g_map_mutex;
+}  // namespace
+
 cb_status cb_attn_launch_tensor(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t st) {
     (void)ctx;
     if (p.P != 16) return CB_ERR_UNSUPPORTED;
+    const MapKey key = {p.q, p.k_pool, p.v_pool, p.k_tree, p.v_tree, p.D, p.Hq, p.Hkv, p.P, p.T, p.B, p.G, p.NPT, p.num_pages};
     TcMaps maps;
-    if (!encode_map(&maps.k_pool, p.k_pool, p.D, p.Hkv, p.P, p.num_pages, 1, 16)) return CB_ERR_CUDA;
-    if (!encode_map(&maps.v_pool, p.v_pool, p.D, p.Hkv, p.P, p.num_pages, 1, 16)) return CB_ERR_CUDA;
-    if (!encode_map(&maps.k_tree, p.k_tree, p.D, p.Hkv, p.T, p.B, 1, 16)) return CB_ERR_CUDA;
-    if (!encode_map(&maps.v_tree, p.v_tree, p.D, p.Hkv, p.T, p.B, 1, 16)) return CB_ERR_CUDA;
-    if (!encode_map(&maps.q, p.q, p.D, p.Hq, p.T, p.B, p.G, p.NPT)) return CB_ERR_CUDA;
+    bool hit = false;
+    {
+        std::lock_guard<std::mutex> lock(g_map_mutex);
+        for (int i = 0; i < g_map_used && !hit; ++i)
+            if (g_map_keys[i] == key) { maps = g_map_vals[i]; hit = true; }
+    }
+    if (!hit) {
+        if (!encode_map(&maps.k_pool, p.k_pool, p.D, p.Hkv, p.P, p.num_pages, 1, 16)) return CB_ERR_CUDA;
+        if (!encode_map(&maps.v_pool, p.v_pool, p.D, p.Hkv, p.P, p.num_pages, 1, 16)) return CB_ERR_CUDA;
+        if (!encode_map(&maps.k_tree, p.k_tree, p.D, p.Hkv, p.T, p.B, 1, 16)) return CB_ERR_CUDA;
+        if (!encode_map(&maps.v_tree, p.v_tree, p.D, p.Hkv, p.T, p.B, 1, 16)) return CB_ERR_CUDA;
+        if (!encode_map(&maps.q, p.q, p.D, p.Hq, p.T, p.B, p.G, p.NPT)) return CB_ERR_CUDA;
+        std::lock_guard<std::mutex> lock(g_map_mutex);
+        const int slot = g_map_used < kMapCache ? g_map_used++ : (g_map_next++ % kMapCache);
+        g_map_keys[slot] = key;
+        g_map_vals[slot] = maps;
+    }
     return p.D == 128 ? launch<128>(p, maps, st) : launch<64>(p, maps, st);
 }
