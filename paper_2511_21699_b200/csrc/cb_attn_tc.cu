@@ -107,6 +107,11 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
     "+r"(a[29]), "+r"(a[30]), "+r"(a[31])
 // Waits for this thread's outstanding TMEM loads; naming the destination registers keeps their uses below the wait.
 #define CB_TMEM_WAIT_LD32(a) asm volatile("tcgen05.wait::ld.sync.aligned;" : CB_RW32(a) :: "memory")
+#define CB_TMEM_ST16(a, o, taddr)                                                                                    \
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, " \
+                 "%12, %13, %14, %15};" ::"r"(a[o + 0]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]),  \
+                 "r"(a[o + 5]), "r"(a[o + 6]), "r"(a[o + 7]), "r"(a[o + 8]), "r"(a[o + 9]), "r"(a[o + 10]),           \
+                 "r"(a[o + 11]), "r"(a[o + 12]), "r"(a[o + 13]), "r"(a[o + 14]), "r"(a[o + 15]), "r"(taddr) : "memory")
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -535,9 +540,9 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     // pass 2: P = 2^(s * scale - m), written back over S as packed bf16 (64 scores -> 32 columns)
                     const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), negmu2 = f2_pack(-mu, -mu);
                     uint64_t lsa = f2_pack(0.f, 0.f), lsb = f2_pack(0.f, 0.f);
-                    uint32_t pk[32];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
+                        uint32_t pk[16];
                         uint32_t* cur = (c & 1) ? sb : sa;
                         uint32_t* nxt = (c & 1) ? sa : sb;
                         CB_TMEM_WAIT_LD32(cur);
@@ -555,10 +560,10 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                             p0 = ex2(p0); p1 = ex2(p1); p2 = ex2(p2); p3 = ex2(p3);
                             lsa = f2_add(lsa, f2_pack(p0, p1));
                             lsb = f2_add(lsb, f2_pack(p2, p3));
-                            pk[(c & 1) * 16 + (jx >> 1)] = pack_bf16(p0, p1);
-                            pk[(c & 1) * 16 + (jx >> 1) + 1] = pack_bf16(p2, p3);
+                            pk[jx >> 1] = pack_bf16(p0, p1);
+                            pk[(jx >> 1) + 1] = pack_bf16(p2, p3);
                         }
-                        if (c & 1) CB_TMEM_ST32(pk, 0, ts + (c >> 1) * 32);
+                        CB_TMEM_ST16(pk, 0, ts + c * 16);             // the 32 scores just read become 16 columns of packed P
                     }
                     float l0, l1, l2, l3;
                     f2_unpack(lsa, l0, l1);
