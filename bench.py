@@ -250,9 +250,8 @@ def run_ours(args, rank, world, local_rank):
     n_old = dev(np.stack([prefill + ADVANCE * s for s in range(total)]).astype(np.int32))
     n_new = dev(np.stack([prefill + ADVANCE * (s + 1) for s in range(total)]).astype(np.int32))
     cb.cb_update(toks_d, dev(np.zeros(B, np.int32)), dev(prefill))          # prompt initialisation, untimed
-    tree = cb.alloc_tree()
+    trees = [cb.alloc_tree() for _ in range(total)]         # every step keeps its own tree, so later passes can reuse it
     res = cb.alloc_accept()
-    n_nodes_all = torch.zeros(total, B, dtype=torch.int32, device=device)
     if args.full_trees:
         trees = [W.random_tree(cfg.seed, b, T, cfg.max_depth, T) for b in range(B)]
         par, dep = np.stack([t[0] for t in trees]), np.stack([t[1] for t in trees])
@@ -261,20 +260,14 @@ def run_ours(args, rank, world, local_rank):
         ftree = dict(tokens=dev(np.maximum(par, 0)), parent=dev(par), depth=dev(dep), mask=dev(mask.view(np.int32)),
                      n_nodes=dev(nn))
 
-    def step(s, ev=None):
+    def step(s):
         r = s % R
-        tr = dict(tree)
-        tr["n_nodes"] = n_nodes_all[s]
-        if ev: ev[0].record()
+        tr = trees[s]
         cb.cb_update(toks_d, n_old[s], n_new[s])
-        if ev: ev[1].record()
         cb.cb_draft_tree(toks_d, n_new[s], tr)
-        if ev: ev[2].record()
         at = ftree if args.full_trees else tr
         cb.cb_tree_attn(q, kps[r], vps[r], bt_d, ctx_d, kt, vt, at["mask"], at["n_nodes"], out=out, max_ctx=int(ctx.max()))
-        if ev: ev[3].record()
         cb.cb_accept(at, logits=lgs[r], res=res)
-        if ev: ev[4].record()
 
     stream = torch.cuda.Stream(device=device)
     with torch.cuda.stream(stream):
@@ -308,16 +301,48 @@ def run_ours(args, rank, world, local_rank):
             stream.synchronize()
             times.append(e0.elapsed_time(e1))
         ms_total = float(np.median(times))
-        # per-call timing pass (eager, events around every call) for the roofline of the dominant kernel
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(K)]
-        for i, s in enumerate(range(Wm + K, Wm + 2 * K)):
-            step(s, evs[i])
+        nn_timed = torch.stack([t["n_nodes"] for t in trees[Wm:Wm + K]]).cpu().numpy().astype(np.float64)
+        # Per-call times, for the roofline of the dominant kernel: each of the four calls is captured K times back to
+        # back in a graph of its own (inputs rotating as in the step) and the replay is timed with events on this stream.
+        # Eager launches would measure the host's enqueue cost at batch 1, not the kernels.
+        base = Wm + K
+
+        def one_call(which, s):
+            r = s % R
+            tr = trees[s]
+            at = ftree if args.full_trees else tr
+            if which == 0:
+                cb.cb_update(toks_d, n_old[s], n_new[s])
+            elif which == 1:
+                cb.cb_draft_tree(toks_d, n_new[s], tr)
+            elif which == 2:
+                cb.cb_tree_attn(q, kps[r], vps[r], bt_d, ctx_d, kt, vt, at["mask"], at["n_nodes"], out=out, max_ctx=int(ctx.max()))
+            else:
+                cb.cb_accept(at, logits=lgs[r], res=res)
+
+        for s in range(base, base + K):                      # one eager pass leaves valid trees for every step index
+            step(s)
         stream.synchronize()
+        per_med = np.zeros(4)
+        for which in range(4):
+            gc = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gc, stream=stream):
+                for s in range(base, base + K):
+                    one_call(which, s)
+            tt = []
+            for _ in range(3):
+                e0.record(stream)
+                gc.replay()
+                e1.record(stream)
+                stream.synchronize()
+                tt.append(e0.elapsed_time(e1) / K)
+            per_med[which] = float(np.median(tt))
+            del gc
+        nn_percall = torch.stack([t["n_nodes"] for t in trees[base:base + K]]).cpu().numpy().astype(np.float64)
         clocks = sampler.stop()
-    per = np.array([[evs[i][j].elapsed_time(evs[i][j + 1]) for j in range(4)] for i in range(K)])   # ms
-    per_med = np.median(per, axis=0)
-    nn_timed = n_nodes_all[Wm:Wm + K].cpu().numpy().astype(np.float64)
     nn_attn = (np.full((K, B), float(T)) if args.full_trees else nn_timed)
+    if args.full_trees:
+        nn_percall = np.full((K, B), float(T))
     tokens = float(nn_attn.sum())
     if world > 1:
         t = torch.tensor([ms_total], device=device)
@@ -345,7 +370,7 @@ def run_ours(args, rank, world, local_rank):
             dq.copy_(hq, non_blocking=True); dkt.copy_(hkt, non_blocking=True); dvt.copy_(hvt, non_blocking=True)
             dlg.copy_(hlg, non_blocking=True)
             d_old.copy_(h_old[s], non_blocking=True); d_new.copy_(h_new[s], non_blocking=True)
-            tr = dict(tree); tr["n_nodes"] = n_nodes_all[s]
+            tr = trees[s]
             cb.cb_update(toks_d, d_old, d_new)
             cb.cb_draft_tree(toks_d, d_new, tr)
             at = ftree if args.full_trees else tr
@@ -373,7 +398,7 @@ def run_ours(args, rank, world, local_rank):
             dist.destroy_process_group()
         return
     hbm_peak, tf_peak, peak_kind = peaks()
-    nn_mean = nn_attn.mean(axis=0)
+    nn_mean = nn_percall.mean(axis=0)                       # trees of the steps the per-call graphs ran
     a_bytes = attn_bytes(cfg, ctx, nn_mean)
     attn_ms = float(per_med[2])
     t_mem, t_cmp = a_bytes / (hbm_peak * 1e9), attn_flops(cfg, ctx, nn_mean, float(np.sum(nn_mean * 4))) / (tf_peak * 1e12)
@@ -387,7 +412,7 @@ def run_ours(args, rank, world, local_rank):
     else:
         fl = attn_flops(cfg, ctx, nn_mean, float(np.sum(nn_mean * 4)))
         roof = {"bound": "tensor", "achieved": fl / (attn_ms * 1e-3) / 1e12, "peak": tf_peak, "unit": "TFLOP/s"}
-    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": traffic, "kernel": "cb_tree_attn (attention + split combine)",
+    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": traffic, "kernel": "cb_tree_attn (attention kernel + merge pass)",
                  "ms_per_launch": attn_ms, "peak_source": peak_kind + " (MEASURED_PEAKS.json)" if peak_kind == "measured" else "fallback",
                  "algorithmic_bytes": a_bytes})
     line = {
