@@ -246,6 +246,9 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
     const int RT = p.NPT * p.G;                               // rows of a row tile that exist
+    // The merge pass is launched as a programmatic dependent: its blocks may take the SMs that this grid's CTAs leave and
+    // do their set-up there; they wait for this whole grid before they read any partial.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // this CTA's range of the global tile sequence
@@ -678,6 +681,7 @@ __global__ void __launch_bounds__(256) cb_attn_merge_kernel(const CbAttnParams p
     }
     __syncthreads();
     const int nparts = s_nparts;
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // the attention grid has finished and its writes are visible
     const size_t rstride = (size_t)(D + 4), sstride = (size_t)2 * CB_MT * rstride;
     for (int r2 = blockIdx.y * 8 + warp; r2 < nrt * CB_MT; r2 += gridDim.y * 8) {
         const int wg = r2 / CB_MT, row = r2 % CB_MT;
@@ -759,7 +763,15 @@ cb_status launch(const CbAttnParams& p, const TcMaps& maps, cudaStream_t st) {
     }
     cb_attn_tc_kernel<D><<<p.nc, kThreads, Cfg<D>::SMEM_ALLOC, st>>>(p, maps);
     CB_CUDA(cudaGetLastError());
-    cb_attn_merge_kernel<D><<<dim3(p.nc, 4), 256, 0, st>>>(p);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(p.nc, 4); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        CB_CUDA(cudaLaunchKernelEx(&cfg, cb_attn_merge_kernel<D>, p));
+    }
     cb_count_launch(2);
     CB_CUDA(cudaGetLastError());
     return CB_OK;
