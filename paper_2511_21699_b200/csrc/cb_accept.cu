@@ -80,6 +80,7 @@ __global__ void __launch_bounds__(256) cb_accept_logits_kernel(
     const int32_t* __restrict__ n_nodes, unsigned long long* rowmax, uint32_t* ticket,
     int32_t* __restrict__ n_accept, int32_t* __restrict__ accept_nodes, int32_t* __restrict__ out_tokens,
     int32_t* __restrict__ target_out) {
+    CB_PDL_ENTRY();
     const int b = blockIdx.z, i = blockIdx.y, ck = blockIdx.x, tid = threadIdx.x;
     const int n = n_nodes[b];
     __shared__ unsigned long long s_red[8];
@@ -181,6 +182,7 @@ __global__ void __launch_bounds__(128) cb_accept_ids_kernel(int B, int T, int Dm
                                                             const int32_t* __restrict__ dep, const int32_t* __restrict__ n_nodes,
                                                             int32_t* __restrict__ n_accept, int32_t* __restrict__ accept_nodes,
                                                             int32_t* __restrict__ out_tokens, int32_t* __restrict__ target_out) {
+    CB_PDL_ENTRY();
     __shared__ int32_t s_target[4][CB_MAX_T];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int b = blockIdx.x * 4 + w;
@@ -208,9 +210,8 @@ extern "C" cb_status cb_accept(cb_ctx* ctx, const int32_t* tree_tokens, const in
     const int T = c.max_nodes, Dmax = c.max_depth;
     cudaStream_t st = (cudaStream_t)stream;
     if (target_ids_in) {
-        cb_accept_ids_kernel<<<(c.batch + 3) / 4, 128, 0, st>>>(c.batch, T, Dmax, target_ids_in, tree_tokens, tree_parent,
-                                                                 tree_depth, n_nodes, n_accept, accept_nodes, out_tokens,
-                                                                 target_ids_out);
+        CB_CUDA(cb_launch_pdl(cb_accept_ids_kernel, dim3((c.batch + 3) / 4), dim3(128), 0, st, c.batch, T, Dmax, target_ids_in, tree_tokens,
+                              tree_parent, tree_depth, n_nodes, n_accept, accept_nodes, out_tokens, target_ids_out));
     } else {
         CB_CHECK_ARG(logits_dtype == CB_DTYPE_F32 || logits_dtype == CB_DTYPE_BF16);
         CB_CHECK_ARG(logits_row_stride >= c.vocab);
@@ -226,16 +227,15 @@ extern "C" cb_status cb_accept(cb_ctx* ctx, const int32_t* tree_tokens, const in
         dim3 grid(cpr, T, c.batch);
         if (c.batch > 65535) return CB_ERR_UNSUPPORTED;
         if (logits_dtype == CB_DTYPE_F32)
-            cb_accept_logits_kernel<false><<<grid, 256, 0, st>>>(T, c.vocab, Dmax, chunk, cpr, logits, logits_row_stride,
-                                                                 tree_tokens, tree_parent, tree_depth, n_nodes, ctx->d_rowmax,
-                                                                 ctx->d_ticket, n_accept, accept_nodes, out_tokens, target_ids_out);
+            CB_CUDA(cb_launch_pdl(cb_accept_logits_kernel<false>, grid, dim3(256), 0, st, T, c.vocab, Dmax, chunk, cpr, logits, logits_row_stride,
+                                  tree_tokens, tree_parent, tree_depth, n_nodes, ctx->d_rowmax, ctx->d_ticket, n_accept, accept_nodes,
+                                  out_tokens, target_ids_out));
         else
-            cb_accept_logits_kernel<true><<<grid, 256, 0, st>>>(T, c.vocab, Dmax, chunk, cpr, logits, logits_row_stride,
-                                                                tree_tokens, tree_parent, tree_depth, n_nodes, ctx->d_rowmax,
-                                                                ctx->d_ticket, n_accept, accept_nodes, out_tokens, target_ids_out);
+            CB_CUDA(cb_launch_pdl(cb_accept_logits_kernel<true>, grid, dim3(256), 0, st, T, c.vocab, Dmax, chunk, cpr, logits, logits_row_stride,
+                                  tree_tokens, tree_parent, tree_depth, n_nodes, ctx->d_rowmax, ctx->d_ticket, n_accept, accept_nodes,
+                                  out_tokens, target_ids_out));
     }
     cb_count_launch(1);
-    CB_CUDA(cudaGetLastError());
     return CB_OK;
 }
 

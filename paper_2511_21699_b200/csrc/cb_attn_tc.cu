@@ -246,9 +246,9 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
     const int RT = p.NPT * p.G;                               // rows of a row tile that exist
-    // The merge pass is launched as a programmatic dependent: its blocks may take the SMs that this grid's CTAs leave and
-    // do their set-up there; they wait for this whole grid before they read any partial.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // The merge pass (like the next kernel of a step) is launched as a programmatic dependent: its blocks may take the SMs
+    // that this grid's CTAs leave and do their set-up there; they wait for this whole grid before they read any partial.
+    CB_PDL_ENTRY();
 
     if (warp == 0) {
         // this CTA's range of the global tile sequence
@@ -644,6 +644,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
 // and combines the partials that CTA c and the following CTAs left for it.  One warp per output row.
 template <int D>
 __global__ void __launch_bounds__(256) cb_attn_merge_kernel(const CbAttnParams p) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the wait comes below, after the set-up that reads inputs only
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x;
     const long long tot = cb_sched_total(p, lane);
@@ -761,17 +762,8 @@ cb_status launch(const CbAttnParams& p, const TcMaps& maps, cudaStream_t st) {
         CB_CUDA(cudaFuncSetAttribute(cb_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<D>::SMEM_ALLOC));
         attr_set = true;
     }
-    cb_attn_tc_kernel<D><<<p.nc, kThreads, Cfg<D>::SMEM_ALLOC, st>>>(p, maps);
-    CB_CUDA(cudaGetLastError());
-    {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(p.nc, 4); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = st;
-        cudaLaunchAttribute at[1];
-        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        at[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = at; cfg.numAttrs = 1;
-        CB_CUDA(cudaLaunchKernelEx(&cfg, cb_attn_merge_kernel<D>, p));
-    }
+    CB_CUDA(cb_launch_pdl(cb_attn_tc_kernel<D>, dim3(p.nc), dim3(kThreads), Cfg<D>::SMEM_ALLOC, st, p, maps));
+    CB_CUDA(cb_launch_pdl(cb_attn_merge_kernel<D>, dim3(p.nc, 4), dim3(256), 0, st, p));
     cb_count_launch(2);
     CB_CUDA(cudaGetLastError());
     return CB_OK;

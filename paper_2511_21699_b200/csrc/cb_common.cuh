@@ -91,6 +91,28 @@ void cb_count_launch(int n);
 
 #define CB_ATTN_MAX_UNITS 640   // partial row tiles (128 rows x (D + 4) floats): 2 shared units x 2 row tiles per persistent CTA, 160 CTAs
 
+// Programmatic dependent launch.  Every kernel of the step begins with CB_PDL_ENTRY: it waits until the kernels before
+// it in the stream have finished (so nothing they wrote or still read is touched early) and then lets the next kernel's
+// blocks be scheduled as SMs become free, which hides launch latency between the microsecond-scale kernels of a step.
+#define CB_PDL_ENTRY()                                               \
+    do {                                                             \
+        asm volatile("griddepcontrol.wait;" ::: "memory");           \
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); \
+    } while (0)
+#ifdef __CUDACC__
+#include <utility>
+template <typename... KArgs, typename... Args>
+inline cudaError_t cb_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#endif
+
 #define CB_CHECK_ARG(cond) do { if (!(cond)) return CB_ERR_INVALID_ARG; } while (0)
 #include <stdio.h>
 // CUDA failures are exceptional: say where and what on stderr, then report CB_ERR_CUDA.

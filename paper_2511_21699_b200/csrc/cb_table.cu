@@ -150,6 +150,7 @@ __global__ void __launch_bounds__(128) cb_update_kernel(CbTables t, int B, const
                                                         int64_t row_stride, const int32_t* __restrict__ n_old,
                                                         const int32_t* __restrict__ n_new, uint32_t* status,
                                                         unsigned long long* counters) {
+    CB_PDL_ENTRY();
     const int lane = threadIdx.x & 31;
     const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (b >= B) return;
@@ -194,6 +195,7 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, int T, int cr
                                                        int32_t* __restrict__ o_dep, uint32_t* __restrict__ o_mask,
                                                        int32_t* __restrict__ o_n, uint32_t* status,
                                                        unsigned long long* counters) {
+    CB_PDL_ENTRY();
     extern __shared__ int32_t smem[];
     DraftSmem S;
     S.tok = smem; S.par = S.tok + T; S.dep = S.par + T;
@@ -325,10 +327,9 @@ extern "C" cb_status cb_update(cb_ctx* ctx, const int32_t* tokens, int64_t row_s
                                const int32_t* n_new, void* stream) {
     CB_CHECK_ARG(ctx && tokens && n_old && n_new && row_stride >= 1);
     const int B = ctx->cfg.batch, wpb = 4;
-    cb_update_kernel<<<(B + wpb - 1) / wpb, wpb * 32, 0, (cudaStream_t)stream>>>(
-        ctx->tables, B, tokens, row_stride, n_old, n_new, ctx->d_status, ctx->d_counters);
+    CB_CUDA(cb_launch_pdl(cb_update_kernel, dim3((B + wpb - 1) / wpb), dim3(wpb * 32), 0, (cudaStream_t)stream, ctx->tables, B, tokens, row_stride,
+                          n_old, n_new, ctx->d_status, ctx->d_counters));
     cb_count_launch(1);
-    CB_CUDA(cudaGetLastError());
     return CB_OK;
 }
 
@@ -343,10 +344,8 @@ extern "C" cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t r
     const size_t smem = sizeof(int32_t) * ((size_t)3 * T + (size_t)6 * NL + (size_t)NL * c.FL * c.FC);
     if (smem > 48 * 1024) return CB_ERR_UNSUPPORTED;
     const int threads = 32 * max(1, min(8, NL));
-    cb_draft_kernel<<<c.batch, threads, smem, (cudaStream_t)stream>>>(
-        ctx->tables, T, c.crt, c.max_depth, NL, tokens, row_stride, seq_len, tree_tokens, tree_parent,
-        tree_depth, tree_mask, n_nodes, ctx->d_status, ctx->d_counters);
+    CB_CUDA(cb_launch_pdl(cb_draft_kernel, dim3(c.batch), dim3(threads), smem, (cudaStream_t)stream, ctx->tables, T, c.crt, c.max_depth, NL, tokens,
+                          row_stride, seq_len, tree_tokens, tree_parent, tree_depth, tree_mask, n_nodes, ctx->d_status, ctx->d_counters));
     cb_count_launch(1);
-    CB_CUDA(cudaGetLastError());
     return CB_OK;
 }
