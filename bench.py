@@ -38,6 +38,22 @@ def parse():
     return ap.parse_args()
 
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one cb_attn_tc_kernel launch, from the ncu capture
+# summarised in profiles/cb_attn_tc_kernel_<workload>.md.  It is reported only while the kernel sources still hash to the
+# captured ones; after any change to them the figure is stale and `traffic` is null until the capture is redone.
+ATTN_TRAFFIC = {"sources_sha1": "31a9ea0abde9f32d328318baf033ae54640fa3b4",
+                "bytes_per_launch": {"c2_7b": 70.35e6, "c3_8b_gqa": 594.6e6, "c4_13b_turns": 2806.9e6}}
+
+
+def attn_sources_sha1():
+    import hashlib
+    h = hashlib.sha1()
+    for f in ("cb_attn_tc.cu", "cb_attn.cuh", "cb_attn.cu"):
+        with open(os.path.join(ROOT, "paper_2511_21699_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -253,8 +269,8 @@ def run_ours(args, rank, world, local_rank):
     trees = [cb.alloc_tree() for _ in range(total)]         # every step keeps its own tree, so later passes can reuse it
     res = cb.alloc_accept()
     if args.full_trees:
-        trees = [W.random_tree(cfg.seed, b, T, cfg.max_depth, T) for b in range(B)]
-        par, dep = np.stack([t[0] for t in trees]), np.stack([t[1] for t in trees])
+        rtrees = [W.random_tree(cfg.seed, b, T, cfg.max_depth, T) for b in range(B)]
+        par, dep = np.stack([t[0] for t in rtrees]), np.stack([t[1] for t in rtrees])
         mask = np.stack([W.tree_mask_from_parents(par[b], T, (T + 31) // 32) for b in range(B)])
         nn = np.full(B, T, np.int32)
         ftree = dict(tokens=dev(np.maximum(par, 0)), parent=dev(par), depth=dev(dep), mask=dev(mask.view(np.int32)),
@@ -402,11 +418,7 @@ def run_ours(args, rank, world, local_rank):
     a_bytes = attn_bytes(cfg, ctx, nn_mean)
     attn_ms = float(per_med[2])
     t_mem, t_cmp = a_bytes / (hbm_peak * 1e9), attn_flops(cfg, ctx, nn_mean, float(np.sum(nn_mean * 4))) / (tf_peak * 1e12)
-    traffic = None
-    tp = os.path.join(ROOT, "profiles", "attn_traffic.json")
-    if os.path.exists(tp):
-        with open(tp) as f:
-            traffic = json.load(f).get(cfg.name)
+    traffic = ATTN_TRAFFIC["bytes_per_launch"].get(cfg.name) if ATTN_TRAFFIC["sources_sha1"] == attn_sources_sha1() else None
     if t_mem >= t_cmp:
         roof = {"bound": "hbm", "achieved": a_bytes / (attn_ms * 1e-3) / 1e9, "peak": hbm_peak, "unit": "GB/s"}
     else:
