@@ -5,7 +5,9 @@
 // pair of 128-row tiles (row = node_local * G + g, NPT = 128 / G nodes per tile), or a single tile when
 // the whole tree fits one tile; only row tiles that hold valid nodes form units.  All units, in
 // (sequence, kv head, row group) order, laid end to end give one global sequence of key tiles; it is cut
-// into `nc` equal ranges, one per persistent CTA (a stream-K split).  A CTA therefore finishes whole
+// into `nc` equal ranges, one per persistent CTA (a stream-K split).  Starting a unit costs about as much as two or
+// three tiles (query load, pipeline refill, epilogue), so every unit is preceded by that many padding positions in the
+// sequence: they carry no work, they only make a CTA that handles many short units receive fewer tiles.  A CTA therefore finishes whole
 // units, plus at most one unit it shares with earlier CTAs and one it shares with later CTAs; shared
 // units leave unnormalised partials that the merge pass combines.
 #pragma once
@@ -38,7 +40,8 @@ struct CbAttnParams {
 // Per-sequence shape of the decomposition.
 struct CbSeqShape {
     int n, ctx, tiles, mtn, RG;
-    long long W;          // key tiles of all units of this sequence
+    int ov;               // padding positions in front of each unit of this sequence
+    long long W;          // positions (padding + key tiles) of all units of this sequence
 };
 
 __device__ __forceinline__ CbSeqShape cb_seq_shape(const CbAttnParams& p, int b) {
@@ -48,7 +51,8 @@ __device__ __forceinline__ CbSeqShape cb_seq_shape(const CbAttnParams& p, int b)
     s.tiles = (s.ctx + CB_KT - 1) / CB_KT + 1;
     s.mtn = (s.n + p.NPT - 1) / p.NPT;
     s.RG = p.MT == 1 ? (s.mtn > 0 ? 1 : 0) : (s.mtn + 1) / 2;
-    s.W = (long long)p.Hkv * s.RG * s.tiles;
+    s.ov = s.mtn >= 2 ? 3 : 2;
+    s.W = (long long)p.Hkv * s.RG * (s.tiles + s.ov);
     return s;
 }
 
@@ -96,7 +100,7 @@ __device__ __forceinline__ void cb_sched_locate(const CbAttnParams& p, long long
     *pre_out = fpre;
 }
 
-// One unit's share of a CTA's range.
+// One unit's share of a CTA's range: key tiles [t0, t1) of the unit's `tiles`.
 struct CbUnit {
     int b, kh, rg, t0, t1, tiles, n, ctx, nrt;   // nrt = valid row tiles in the group (1 or 2)
 };
@@ -111,17 +115,22 @@ struct CbWalker {
         if (g < g1) s = cb_seq_shape(p, b);
     }
     __device__ __forceinline__ bool next(const CbAttnParams& p, CbUnit* u) {
-        if (g >= g1) return false;
-        while (g >= pre + s.W) { pre += s.W; ++b; s = cb_seq_shape(p, b); }
-        const long long off = g - pre;
-        const int j = (int)(off / s.tiles);
-        u->t0 = (int)(off - (long long)j * s.tiles);
-        const long long room = g1 - g;
-        u->t1 = (int)min((long long)s.tiles, (long long)u->t0 + room);
-        u->b = b; u->kh = j / s.RG; u->rg = j % s.RG; u->tiles = s.tiles; u->n = s.n; u->ctx = s.ctx;
-        u->nrt = p.MT == 1 ? 1 : min(2, s.mtn - 2 * u->rg);
-        g += u->t1 - u->t0;
-        return true;
+        while (true) {
+            if (g >= g1) return false;
+            while (g >= pre + s.W) { pre += s.W; ++b; s = cb_seq_shape(p, b); }
+            const long long off = g - pre;
+            const int vt = s.tiles + s.ov;                    // positions of one unit
+            const int j = (int)(off / vt);
+            const int v0 = (int)(off - (long long)j * vt);
+            const int v1 = (int)min((long long)vt, (long long)v0 + (g1 - g));
+            g += v1 - v0;
+            u->t0 = max(v0 - s.ov, 0);
+            u->t1 = max(v1 - s.ov, 0);
+            if (u->t1 <= u->t0) continue;                     // only padding of this unit falls into the range
+            u->b = b; u->kh = j / s.RG; u->rg = j % s.RG; u->tiles = s.tiles; u->n = s.n; u->ctx = s.ctx;
+            u->nrt = p.MT == 1 ? 1 : min(2, s.mtn - 2 * u->rg);
+            return true;
+        }
     }
 };
 

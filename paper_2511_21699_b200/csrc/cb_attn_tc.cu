@@ -656,11 +656,13 @@ __global__ void __launch_bounds__(256) cb_attn_merge_kernel(const CbAttnParams p
     cb_sched_locate(p, g1 - 1, lane, &b, &pre);
     const CbSeqShape s = cb_seq_shape(p, b);
     const long long off = g1 - 1 - pre;
-    const int j = (int)(off / s.tiles);
-    if ((int)(off - (long long)j * s.tiles) == s.tiles - 1) return;   // the unit ends with this range
-    const long long ustart = pre + (long long)j * s.tiles;
-    if (ustart < g0) return;                                  // started by an earlier CTA: that CTA's block merges it
-    const int c_last = cb_cta_of(tot, p.nc, ustart + s.tiles - 1);
+    const int vt = s.tiles + s.ov;                            // positions of one unit: padding, then its key tiles
+    const int j = (int)(off / vt);
+    if ((int)(off - (long long)j * vt) == vt - 1) return;     // the unit ends with this range
+    const long long ustart = pre + (long long)j * vt, first_tile = ustart + s.ov;
+    if (first_tile < g0) return;                              // started by an earlier CTA: that CTA's block merges it
+    if (first_tile >= g1) return;                             // only padding so far: the next CTA starts the unit
+    const int c_last = cb_cta_of(tot, p.nc, ustart + vt - 1);
     const int kh = j / s.RG, rg = j % s.RG;
     const int nrt = p.MT == 1 ? 1 : min(2, s.mtn - 2 * rg);
     const int RT = p.NPT * p.G;
