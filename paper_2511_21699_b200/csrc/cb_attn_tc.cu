@@ -112,6 +112,12 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
                  "%12, %13, %14, %15};" ::"r"(a[o + 0]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]),  \
                  "r"(a[o + 5]), "r"(a[o + 6]), "r"(a[o + 7]), "r"(a[o + 8]), "r"(a[o + 9]), "r"(a[o + 10]),           \
                  "r"(a[o + 11]), "r"(a[o + 12]), "r"(a[o + 13]), "r"(a[o + 14]), "r"(a[o + 15]), "r"(taddr) : "memory")
+// 32-byte store: one instruction fills a whole DRAM sector of this thread's output row
+__device__ __forceinline__ void st_global_v8(void* ptr, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t a4, uint32_t a5, uint32_t a6,
+                                             uint32_t a7) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(ptr), "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(a4), "r"(a5), "r"(a6),
+                 "r"(a7) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -332,12 +338,16 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                 auto issue_pv = [&](int ol, int buf, uint32_t vslot, bool accum) {
                     mma_pv_block(tmem + C::O_COL + ol * D, tmem + buf * 128, v_lo0 + vslot * (C::TILE_BYTES >> 4), idesc_o, accum ? 1u : 0u);
                 };
-                while (ok && wk.next(p, &u)) {
+                CbUnit un;
+                    bool have = wk.next(p, &un);
+                while (ok && have) {
+                    u = un;
                     const bool two = u.nrt == 2;
                     if (!(ok = mbar_wait(bar_qfull, uq & 1, s_abort, p.status))) break;
                     tc_fence_after();
                     const uint32_t seq0 = seq;
                     for (int i = u.t0; ok && i <= u.t1; ++i) {
+                        if (i == u.t1) have = wk.next(p, &un);   // its loads overlap the wait for the last P
                         const uint32_t kseq = seq0 + 2 * (i - u.t0), vseq_prev = kseq - 1;
                         const uint32_t ks = kseq % C::NSLOT, vs = vseq_prev % C::NSLOT;
                         if (two) {
@@ -437,7 +447,29 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
         uint32_t c_s0 = 0;                                    // completions of s_full0 consumed so far (warpgroup 0 only)
         uint32_t seq = 0;                                     // ring sequence number of the next unit's first K tile
         bool ok = true;
-        while (ok && wk.next(p, &u)) {
+        // The next unit's shape and this row's ancestor bits are fetched while the current unit is still being finished,
+        // so that their memory round trips do not sit between two units.
+        CbUnit un;
+        uint32_t mrow_n[4] = {0u, 0u, 0u, 0u};
+        auto fetch_next = [&]() {
+            const bool have = wk.next(p, &un);
+            mrow_n[0] = mrow_n[1] = mrow_n[2] = mrow_n[3] = 0u;
+            if (have && (wg == 0 || un.nrt == 2)) {
+                const int nnode = (un.rg * 2 + wg) * p.NPT + row / p.G;
+                if (row < RT && nnode < un.n) {
+                    const uint32_t* mp = p.tree_mask + ((size_t)un.b * p.T + nnode) * p.W;
+                    mrow_n[0] = mp[0];
+                    if (p.W > 1) mrow_n[1] = mp[1];
+                    if (p.W > 2) mrow_n[2] = mp[2];
+                    if (p.W > 3) mrow_n[3] = mp[3];
+                }
+            }
+            return have;
+        };
+        bool have = fetch_next();
+        while (ok && have) {
+            u = un;
+            const uint32_t mrow[4] = {mrow_n[0], mrow_n[1], mrow_n[2], mrow_n[3]};
             const bool two = u.nrt == 2;
             const int nt = u.t1 - u.t0;
             const uint32_t seq0 = seq;
@@ -450,6 +482,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     const uint32_t kseq = seq0 + 2u * (uint32_t)(i - u.t0);
                     ok = mbar_wait(bar_free(kseq % C::NSLOT), (kseq / C::NSLOT) & 1, s_abort, p.status);
                 }
+                have = fetch_next();
                 continue;
             }
             // S(i) is done when tile i's K slot is released (or, for row tile 0 of two, when s_full0 completes);
@@ -463,14 +496,6 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             const bool row_valid = row < RT && node < u.n;
             const bool warp_active = (wq * 32) < RT && (rt * p.NPT + (wq * 32) / p.G) < u.n;   // row 0 of the warp is valid
             const int nct = u.tiles - 1;
-            uint32_t mrow[4] = {0u, 0u, 0u, 0u};
-            if (row_valid) {
-                const uint32_t* mp = p.tree_mask + ((size_t)u.b * p.T + node) * p.W;
-                mrow[0] = mp[0];
-                if (p.W > 1) mrow[1] = mp[1];
-                if (p.W > 2) mrow[2] = mp[2];
-                if (p.W > 3) mrow[3] = mp[3];
-            }
             float m_used = -INFINITY, l = 0.f;
             for (int i = u.t0; i < u.t1; ++i) {
                 const int buf = two ? wg : ((i - u.t0) & 1);
@@ -578,6 +603,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                 mbar_arrive(bar_pready(buf));
             }
             if (!ok) break;
+            have = fetch_next();
             // ---- epilogue of this unit's share: O is complete once its last PV has finished
             if (!(ok = wait_pv(u.t1 - 1))) break;
             tc_fence_after();
@@ -591,16 +617,12 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                         CB_TMEM_LD32(o, 0, tm_O + c * 32);
                         tmem_wait_ld();
                         if (row_valid) {
-                            uint4* op = reinterpret_cast<uint4*>(p.out + (((size_t)u.b * p.T + node) * p.Hq + h) * D + c * 32);
+                            __nv_bfloat16* op = p.out + (((size_t)u.b * p.T + node) * p.Hq + h) * D + c * 32;
+                            uint32_t w[16];
 #pragma unroll
-                            for (int v4 = 0; v4 < 4; ++v4) {
-                                uint4 w;
-                                w.x = pack_bf16(__uint_as_float(o[v4 * 8 + 0]) * inv, __uint_as_float(o[v4 * 8 + 1]) * inv);
-                                w.y = pack_bf16(__uint_as_float(o[v4 * 8 + 2]) * inv, __uint_as_float(o[v4 * 8 + 3]) * inv);
-                                w.z = pack_bf16(__uint_as_float(o[v4 * 8 + 4]) * inv, __uint_as_float(o[v4 * 8 + 5]) * inv);
-                                w.w = pack_bf16(__uint_as_float(o[v4 * 8 + 6]) * inv, __uint_as_float(o[v4 * 8 + 7]) * inv);
-                                op[v4] = w;
-                            }
+                            for (int k2 = 0; k2 < 16; ++k2) w[k2] = pack_bf16(__uint_as_float(o[2 * k2]) * inv, __uint_as_float(o[2 * k2 + 1]) * inv);
+                            st_global_v8(op, w[0], w[1], w[2], w[3], w[4], w[5], w[6], w[7]);
+                            st_global_v8(op + 16, w[8], w[9], w[10], w[11], w[12], w[13], w[14], w[15]);
                         }
                     }
                     if (row_valid && p.lse)
@@ -614,6 +636,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                         CB_TMEM_LD32(o, 0, tm_O + c * 32);
                         tmem_wait_ld();
                         if (row_valid) {
+                            // partial rows are D + 4 floats long: 16-byte aligned only
 #pragma unroll
                             for (int v4 = 0; v4 < 8; ++v4)
                                 *reinterpret_cast<uint4*>(pp + c * 32 + v4 * 4) = make_uint4(o[v4 * 4], o[v4 * 4 + 1], o[v4 * 4 + 2], o[v4 * 4 + 3]);
