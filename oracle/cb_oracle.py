@@ -176,3 +176,31 @@ def tree_attn_rows(q, k_pool, v_pool, block_table, ctx_len, k_tree, v_tree, tree
                              T, Hq, Hkv, D, P, bt.shape[1], float(scale if scale is not None else D ** -0.5),
                              _p(rows), rows.shape[0], _p(out), _p(lse))
     return out, lse
+
+
+def kv_commit(k_pool, v_pool, block_table, ctx_len, k_tree, v_tree, n_accept, accept_nodes):
+    """KV commit of the accepted path (paper Section 3.2: the tokens fed to the verification pass without a cached
+    K/V are the non-KV-cached tokens; once a branch is accepted, its tokens are ordinary context for the next step).
+
+    Per sequence b with m = n_accept[b]: the tree root (node 0, the one pending token) and the m accepted nodes
+    accept_nodes[b, :m], in path order, become context tokens ctx_len[b] .. ctx_len[b] + m: their K and V rows are
+    written into the paged cache at those positions (page block_table[b, pos // P], slot pos % P) and ctx_len[b]
+    grows by m + 1.  The bonus token has no K/V yet; it is the next step's root.  A sequence whose new length would
+    exceed its pages is left untouched.  Arrays: k_pool, v_pool [num_pages, P, Hkv, D] (any dtype; modified in place),
+    k_tree, v_tree [B, T, Hkv, D].  Returns the new ctx_len (int32 [B])."""
+    B = block_table.shape[0]
+    P = k_pool.shape[1]
+    out = np.array(ctx_len, dtype=np.int32, copy=True)
+    for b in range(B):
+        m = int(n_accept[b])
+        ctx = int(ctx_len[b])
+        if m < 0 or ctx + m + 1 > block_table.shape[1] * P:
+            continue
+        path = [0] + [int(x) for x in accept_nodes[b, :m]]
+        for j, node in enumerate(path):
+            pos = ctx + j
+            page = int(block_table[b, pos // P])
+            k_pool[page, pos % P] = k_tree[b, node]
+            v_pool[page, pos % P] = v_tree[b, node]
+        out[b] = ctx + m + 1
+    return out
