@@ -45,7 +45,8 @@ typedef enum {
     CB_ERR_PROBE_LIMIT = 4, /* device: a hash probe visited every bucket without finding a free slot  */
     CB_ERR_TIMEOUT = 5,     /* device: a bounded wait (mbarrier / flag) ran out                        */
     CB_ERR_UNSUPPORTED = 6,
-    CB_ERR_STATIC_LIMIT = 7 /* cb_accept_static: the problem does not fit the built-in scratch array        */
+    CB_ERR_STATIC_LIMIT = 7, /* cb_accept_static: the problem does not fit the built-in scratch array       */
+    CB_ERR_KV_FULL = 8       /* device: cb_kv_commit found a sequence whose pages cannot hold the new tokens   */
 } cb_status;
 
 enum { CB_DTYPE_F32 = 0, CB_DTYPE_BF16 = 1 };
@@ -188,6 +189,36 @@ cb_status cb_accept(cb_ctx* ctx, const int32_t* tree_tokens, const int32_t* tree
                     int32_t logits_dtype, int64_t logits_row_stride, const int32_t* target_ids_in,
                     int32_t* n_accept, int32_t* accept_nodes, int32_t* out_tokens,
                     int32_t* target_ids_out, void* stream);
+
+/*
+ * KV commit of the accepted path (Section 3.2: the draft tokens and the pending token are the tokens of the
+ * verification pass that have no cached K/V; once a branch is accepted its tokens are ordinary context for the next
+ * step).  For every sequence b with m = n_accept[b], the tree root (node 0) and the accepted nodes accept_nodes[b, 0..m),
+ * in that order, become context tokens ctx_len[b] .. ctx_len[b] + m: their rows of k_tree / v_tree are copied into the
+ * paged cache (page block_table[b, pos / P], slot pos % P) and ctx_len[b] grows by m + 1.  The bonus token of cb_accept
+ * has no K/V yet: it is the next step's root.
+ *   k_pool, v_pool  bf16 [num_pages, P, Hkv, D]   written
+ *   block_table     int32 [batch, max_pages]      must already name pages for the new positions
+ *   ctx_len         int32 [batch]                 read and updated in place
+ *   k_tree, v_tree  bf16 [batch, T, Hkv, D]
+ *   n_accept        int32 [batch], accept_nodes int32 [batch, max_depth]   as written by cb_accept
+ * A sequence with ctx_len + m + 1 > max_pages * P is left untouched and CB_ERR_KV_FULL is recorded in the device status;
+ * a node or page index outside its tensor is skipped and recorded as CB_ERR_INVALID_ARG.  Only enqueues work.
+ */
+typedef struct {
+    void* k_pool;
+    void* v_pool;
+    const int32_t* block_table;
+    int32_t* ctx_len;
+    const void* k_tree;
+    const void* v_tree;
+    const int32_t* n_accept;
+    const int32_t* accept_nodes;
+    int32_t max_pages;
+    int32_t num_pages;
+} cb_kv_commit_args;
+
+cb_status cb_kv_commit(cb_ctx* ctx, const cb_kv_commit_args* args, void* stream);
 
 /*
  * cb_accept_static — cb_accept (logits form) for callers that must not allocate device memory.

@@ -10,18 +10,24 @@ CB_OK = 0
 CB_DTYPE_F32, CB_DTYPE_BF16 = 0, 1
 CB_FLAG_NO_FOLLOWER_REFRESH, CB_FLAG_ATTN_CUDA_CORES = 1, 2
 CB_ERR_STATIC_LIMIT = 7
+CB_ERR_KV_FULL = 8
 CB_STATIC_MAX_BATCH, CB_STATIC_MAX_ROWS = 1024, 8192
 CB_NUM_COUNTERS = 8
 COUNTER_NAMES = ["inserts", "leader_evictions", "follower_evictions", "queries", "query_hits", "max_probe"]
 
 EXPORTS = ["cb_workspace_bytes", "cb_create", "cb_destroy", "cb_reset", "cb_update", "cb_draft_tree",
            "cb_tree_attn", "cb_accept", "cb_table_dump", "cb_table_load", "cb_poll_status", "cb_launch_count",
-           "cb_status_str", "cb_accept_static"]
+           "cb_status_str", "cb_accept_static", "cb_kv_commit"]
 
 
 class CbConfigC(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("batch", "LL", "FL", "LC", "FC", "max_nodes", "crt", "max_depth", "vocab",
                                           "n_q_heads", "n_kv_heads", "head_dim", "page_size")] + [("flags", C.c_uint32)]
+
+
+class CbKvCommitArgsC(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("k_pool", "v_pool", "block_table", "ctx_len", "k_tree", "v_tree", "n_accept",
+                                          "accept_nodes")] + [("max_pages", C.c_int32), ("num_pages", C.c_int32)]
 
 
 class CbAttnArgsC(C.Structure):
@@ -50,6 +56,7 @@ def load():
     L.cb_update.argtypes = [vp, vp, i64, vp, vp, vp]
     L.cb_draft_tree.argtypes = [vp, vp, i64, vp, vp, vp, vp, vp, vp, vp]
     L.cb_tree_attn.argtypes = [vp, C.POINTER(CbAttnArgsC), vp]
+    L.cb_kv_commit.argtypes = [vp, C.POINTER(CbKvCommitArgsC), vp]
     L.cb_accept.argtypes = [vp, vp, vp, vp, vp, vp, i32, i64, vp, vp, vp, vp, vp, vp]
     L.cb_accept_static.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, i64, vp, vp, vp, vp, vp]
     L.cb_table_dump.argtypes = [vp, i32, C.POINTER(i32), vp, vp, vp]

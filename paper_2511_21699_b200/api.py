@@ -9,7 +9,7 @@ import numpy as np
 import torch
 
 from . import _lib
-from ._lib import CbConfigC, CbAttnArgsC
+from ._lib import CbConfigC, CbAttnArgsC, CbKvCommitArgsC
 
 
 class CachebackError(RuntimeError):
@@ -137,6 +137,12 @@ class Cacheback:
                         int(max_ctx), float(scale))
         _check(self.lib.cb_tree_attn(self._h, C.byref(a), _stream(stream)), "cb_tree_attn")
         return out
+
+    def cb_kv_commit(self, k_pool, v_pool, block_table, ctx_len, k_tree, v_tree, n_accept, accept_nodes, stream=None):
+        a = CbKvCommitArgsC(_ptr(k_pool, torch.bfloat16), _ptr(v_pool, torch.bfloat16), _ptr(block_table, torch.int32),
+                            _ptr(ctx_len, torch.int32), _ptr(k_tree, torch.bfloat16), _ptr(v_tree, torch.bfloat16),
+                            _ptr(n_accept, torch.int32), _ptr(accept_nodes, torch.int32), block_table.shape[1], k_pool.shape[0])
+        _check(self.lib.cb_kv_commit(self._h, C.byref(a), _stream(stream)), "cb_kv_commit")
 
     def alloc_accept(self):
         B, Dm = self.cfg.batch, self.cfg.max_depth

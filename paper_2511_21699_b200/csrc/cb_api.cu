@@ -216,6 +216,7 @@ extern "C" const char* cb_status_str(cb_status s) {
         case CB_ERR_TIMEOUT: return "bounded device wait ran out";
         case CB_ERR_UNSUPPORTED: return "unsupported device or shape";
         case CB_ERR_STATIC_LIMIT: return "problem larger than the built-in static scratch (see cb_accept_static)";
+        case CB_ERR_KV_FULL: return "a sequence's pages cannot hold the committed tokens";
     }
     return "unknown status";
 }
