@@ -107,6 +107,18 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def reduce_over_ranks(seconds, units, device):
+    """Whole-job figures of a replicated run: the slowest rank's time and the units of all ranks together.
+    (No collective is on the data path: ranks are independent replicas; these two all-reduces only gather the result.)"""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([seconds], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    u = torch.tensor([units], device=device, dtype=torch.float64)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
 def attn_bytes(cfg, ctx, n_nodes):
     """Algorithmic HBM bytes of one cb_tree_attn launch: cached K and V once, tree K/V, Q in, O out."""
     D, Hkv, Hq = cfg.head_dim, cfg.n_kv_heads, cfg.n_q_heads
@@ -360,13 +372,9 @@ def run_ours(args, rank, world, local_rank):
     if args.full_trees:
         nn_percall = np.full((K, B), float(T))
     tokens = float(nn_attn.sum())
+    local_tokens = tokens
     if world > 1:
-        t = torch.tensor([ms_total], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-        tk = torch.tensor([tokens], device=device, dtype=torch.float64)
-        dist.all_reduce(tk, op=dist.ReduceOp.SUM)
-        tokens = float(tk.item())
+        ms_total, tokens = reduce_over_ranks(ms_total, tokens, device)
     value = tokens / (ms_total * 1e-3)
 
     # end to end through the public API with host buffers: H2D of the step's inputs, D2H of its result
@@ -400,11 +408,9 @@ def run_ours(args, rank, world, local_rank):
         for s in range(Wm, Wm + K):
             e2e_step(s)
         e2e_s = time.perf_counter() - t0
-    e2e_tokens = tokens if world == 1 else tokens
+    e2e_tokens = local_tokens
     if world > 1:
-        t = torch.tensor([e2e_s], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+        e2e_s, e2e_tokens = reduce_over_ranks(e2e_s, local_tokens, device)
     e2e_val = e2e_tokens / e2e_s
 
     st, counters = cb.cb_poll_status()
