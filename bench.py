@@ -74,7 +74,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.th = threading.Thread(target=self._read, daemon=True)
             self.th.start()
@@ -318,16 +318,18 @@ def run_ours(args, rank, world, local_rank):
         sampler = ClockSampler(local_rank)
         sampler.start()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = 3
         torch.cuda.synchronize()
-        t_best = None
         times = []
-        for _ in range(reps):
+        reps = 3
+        while len(times) < reps:
             e0.record(stream)
             g.replay()
             e1.record(stream)
             stream.synchronize()
             times.append(e0.elapsed_time(e1))
+            if len(times) == 3:
+                # keep replaying until the timed region spans about 0.4 s, so that the clock sampler sees it
+                reps = int(min(400, max(3, 400.0 / max(float(np.median(times)), 1e-3))))
         ms_total = float(np.median(times))
         nn_timed = torch.stack([t["n_nodes"] for t in trees[Wm:Wm + K]]).cpu().numpy().astype(np.float64)
         # Per-call times, for the roofline of the dominant kernel: each of the four calls is captured K times back to
@@ -439,7 +441,7 @@ def run_ours(args, rank, world, local_rank):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "batch": B, "tree_cap": T, "mean_tree_nodes": float(nn_attn.mean()),
                    "context": [int(ctx.min()), int(ctx.max())], "l2": "rotating %d copies of K/V pool and logits (%.0f MB)" %
-                   (R, R * (pool_bytes + logit_bytes) / 1e6), "launch": "CUDA graph of the timed steps",
+                   (R, R * (pool_bytes + logit_bytes) / 1e6), "launch": "CUDA graph of the timed steps, replayed %d times, median" % reps,
                    "trees": "synthetic full" if args.full_trees else "drafted", "parallelism": "replicas x%d" % world},
         "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
