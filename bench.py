@@ -41,8 +41,8 @@ def parse():
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one cb_attn_tc_kernel launch, from the ncu capture
 # summarised in profiles/cb_attn_tc_kernel_<workload>.md.  It is reported only while the kernel sources still hash to the
 # captured ones; after any change to them the figure is stale and `traffic` is null until the capture is redone.
-ATTN_TRAFFIC = {"sources_sha1": "31a9ea0abde9f32d328318baf033ae54640fa3b4",
-                "bytes_per_launch": {"c2_7b": 70.35e6, "c3_8b_gqa": 594.6e6, "c4_13b_turns": 2806.9e6}}
+ATTN_TRAFFIC = {"sources_sha1": "3b0af9cc8abea278d1aafd0e767d0652980f9456",
+                "bytes_per_launch": {"c2_7b": 70.08e6, "c3_8b_gqa": 589.2e6, "c4_13b_turns": 2792.1e6}}
 
 
 def attn_sources_sha1():
