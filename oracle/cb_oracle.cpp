@@ -8,6 +8,7 @@
 //   Update ....... Section 3.2 last paragraph + Section 3.3 last paragraph (sliding window over accepted
 //                  tokens / over the prompt)
 //   Draft tree ... Section 3.2 (recursive queries, breadth-first growth, TDL and CRT)
+//   Frozen table . Section 3.3 (a read-only second table, queried after the dynamic one while the size cap allows)
 //   Tree mask .... Section 3.2 (a token attends only to its ancestors)
 //   Attention .... the textbook softmax(q.k * scale) v over the visible keys, in double precision
 //   Acceptance ... Section 3.2 (one more token than the accepted draft tokens; longest verified branch)
@@ -96,6 +97,13 @@ struct Table {
     }
 };
 
+// Section 3.3: the frozen table is filled offline and never changes during decoding; a query returns the
+// stored follower list as it is (reading: most frequent first, the order the builder stored) and has no side effect.
+struct Frozen {
+    int LL, FL;
+    std::map<Key, std::vector<Key>> leaders;
+};
+
 inline double bf16_to_double(uint16_t b) {
     uint32_t u = (uint32_t)b << 16;
     float f;
@@ -174,20 +182,60 @@ int64_t orc_table_dump(void* h, int32_t* leaders, int32_t* nfol, int32_t* follow
 // the sequence is not queried.
 // Outputs are padded with -1 (mask rows with 0) beyond n.  query_log (optional) receives, per issued
 // query, LL key tokens followed by the hit count.  Returns n.
-int orc_draft_tree(void* h, const int32_t* s, int seq_len, int T, int crt, int max_depth,
-                   int32_t* tok, int32_t* par, int32_t* dep, uint32_t* mask, int32_t* query_log,
-                   int32_t* n_queries) {
-    Table* t = (Table*)h;
+// Dual-table form (Section 3.3): when a frozen table is given, the dynamic table forms the tree first, as above;
+// then, if the tree is still below T nodes, growth continues from the frozen table.
+// readings: the frozen pass visits, first in first out, every node at which a follower list can be attached (the
+// root and the last node of every complete follower, in the order they were created), and the ends of the
+// complete followers it adds itself join the queue; a query at the root is issued, and its followers appended,
+// only while the tree has fewer than max(1, T - crt) nodes, any other only while it has fewer than T (the same
+// rule that the dynamic pass follows, whose level 1 is the root alone); frozen followers are appended most
+// frequent first and are not compared with the branches already present; frozen queries neither tick the
+// dynamic table's clock nor touch any recency.  frozen_log (optional): per issued frozen query, LL key tokens
+// followed by the hit count.
+static int draft_impl(Table* t, const Frozen* fz, const int32_t* s, int seq_len, int T, int crt, int max_depth,
+                      int32_t* tok, int32_t* par, int32_t* dep, uint32_t* mask, int32_t* query_log,
+                      int32_t* n_queries, int32_t* frozen_log, int32_t* n_frozen_queries) {
     const int LL = t->LL, FL = t->FL, W = (T + 31) / 32;
     std::fill(tok, tok + T, -1);
     std::fill(par, par + T, -1);
     std::fill(dep, dep + T, -1);
     std::fill(mask, mask + (size_t)T * W, 0u);
-    int nq = 0;
+    int nq = 0, nfq = 0;
     if (n_queries) *n_queries = 0;
+    if (n_frozen_queries) *n_frozen_queries = 0;
     if (seq_len < 1 || T < 1) return 0;
     int n = 1;
     tok[0] = s[seq_len - 1]; par[0] = -1; dep[0] = 0;
+    // key = last LL tokens of sequence[0..seq_len-1) ++ tokens on root->leaf (root = s[seq_len-1])
+    auto make_key = [&](int leaf, Key& key) {
+        bool ok = true;
+        std::vector<int32_t> path;                               // leaf up to root
+        for (int c = leaf; c >= 0; c = par[c]) path.push_back(tok[c]);
+        for (int j = 0; j < LL; j++) {                            // j-th token from the end
+            int32_t v;
+            if (j < (int)path.size()) v = path[j];
+            else {
+                int pos = seq_len - 1 - (j - ((int)path.size() - 1));
+                v = pos >= 0 ? s[pos] : -1;
+            }
+            if (v < 0) ok = false;
+            key[LL - 1 - j] = v;
+        }
+        return ok;
+    };
+    // appends the followers fs below leaf while fewer than cap nodes exist; complete ones are reported through ends
+    auto attach = [&](int leaf, const std::vector<Key>& fs, int cap, std::vector<int>& ends) {
+        for (auto& F : fs) {
+            if (n >= cap) break;
+            int p = leaf, k = 0;
+            for (int j = 0; j < FL; j++) {
+                if (n >= cap || dep[p] >= max_depth) break;
+                tok[n] = F[j]; par[n] = p; dep[n] = dep[p] + 1; p = n; n++; k++;
+            }
+            if (k == FL) ends.push_back(p);
+        }
+    };
+    std::vector<int> points{0};                                  // every node that ever was a frontier leaf
     std::vector<int> frontier{0};
     int level = 1;
     while (!frontier.empty() && n < T) {
@@ -196,42 +244,40 @@ int orc_draft_tree(void* h, const int32_t* s, int seq_len, int T, int crt, int m
         for (int leaf : frontier) {
             if (n >= cap) break;
             if (dep[leaf] >= max_depth) continue;
-            // key = last LL tokens of sequence[0..seq_len-1) ++ tokens on root->leaf (root = s[seq_len-1])
             Key key(LL);
-            bool ok = true;
-            {
-                std::vector<int32_t> path;                       // leaf up to root
-                for (int c = leaf; c >= 0; c = par[c]) path.push_back(tok[c]);
-                for (int j = 0; j < LL; j++) {                    // j-th token from the end
-                    int32_t v;
-                    if (j < (int)path.size()) v = path[j];
-                    else {
-                        int pos = seq_len - 1 - (j - ((int)path.size() - 1));
-                        v = pos >= 0 ? s[pos] : -1;
-                    }
-                    if (v < 0) ok = false;
-                    key[LL - 1 - j] = v;
-                }
-            }
-            if (!ok) continue;
+            if (!make_key(leaf, key)) continue;
             auto fs = t->query(key.data());
             if (query_log) {
                 std::copy(key.begin(), key.end(), query_log + (size_t)nq * (LL + 1));
                 query_log[(size_t)nq * (LL + 1) + LL] = (int32_t)fs.size();
             }
             nq++;
-            for (auto& F : fs) {
-                if (n >= cap) break;
-                int p = leaf, k = 0;
-                for (int j = 0; j < FL; j++) {
-                    if (n >= cap || dep[p] >= max_depth) break;
-                    tok[n] = F[j]; par[n] = p; dep[n] = dep[p] + 1; p = n; n++; k++;
-                }
-                if (k == FL) next.push_back(p);
-            }
+            attach(leaf, fs, cap, next);
         }
+        points.insert(points.end(), next.begin(), next.end());
         frontier.swap(next);
         level++;
+    }
+    if (fz) {
+        for (size_t qi = 0; qi < points.size() && n < T; qi++) {  // the queue grows while it is walked
+            const int leaf = points[qi];
+            const int cap = leaf == 0 ? std::max(1, T - crt) : T;
+            if (n >= cap) continue;
+            if (dep[leaf] >= max_depth) continue;
+            Key key(LL);
+            if (!make_key(leaf, key)) continue;
+            auto it = fz->leaders.find(key);
+            const std::vector<Key> none;
+            const std::vector<Key>& fs = it == fz->leaders.end() ? none : it->second;
+            if (frozen_log) {
+                std::copy(key.begin(), key.end(), frozen_log + (size_t)nfq * (LL + 1));
+                frozen_log[(size_t)nfq * (LL + 1) + LL] = (int32_t)fs.size();
+            }
+            nfq++;
+            std::vector<int> ends;
+            attach(leaf, fs, cap, ends);
+            points.insert(points.end(), ends.begin(), ends.end());
+        }
     }
     // Tree mask: a token attends to itself and its ancestors, root included.
     for (int i = 0; i < n; i++) {
@@ -239,7 +285,34 @@ int orc_draft_tree(void* h, const int32_t* s, int seq_len, int T, int crt, int m
         mask[(size_t)i * W + i / 32] |= 1u << (i % 32);
     }
     if (n_queries) *n_queries = nq;
+    if (n_frozen_queries) *n_frozen_queries = nfq;
     return n;
+}
+
+int orc_draft_tree(void* h, const int32_t* s, int seq_len, int T, int crt, int max_depth,
+                   int32_t* tok, int32_t* par, int32_t* dep, uint32_t* mask, int32_t* query_log,
+                   int32_t* n_queries) {
+    return draft_impl((Table*)h, nullptr, s, seq_len, T, crt, max_depth, tok, par, dep, mask, query_log, n_queries, nullptr, nullptr);
+}
+
+void* orc_frozen_new(int LL, int FL) {
+    Frozen* f = new Frozen();
+    f->LL = LL; f->FL = FL;
+    return f;
+}
+void orc_frozen_free(void* h) { delete (Frozen*)h; }
+// One leader with its nf followers (nf * FL tokens), most frequent first.
+void orc_frozen_add(void* h, const int32_t* L, int nf, const int32_t* followers) {
+    Frozen* f = (Frozen*)h;
+    std::vector<Key> fs;
+    for (int i = 0; i < nf; i++) fs.emplace_back(followers + (size_t)i * f->FL, followers + (size_t)(i + 1) * f->FL);
+    f->leaders[Key(L, L + f->LL)] = std::move(fs);
+}
+int orc_draft_tree_dual(void* h, void* hf, const int32_t* s, int seq_len, int T, int crt, int max_depth,
+                        int32_t* tok, int32_t* par, int32_t* dep, uint32_t* mask, int32_t* query_log,
+                        int32_t* n_queries, int32_t* frozen_log, int32_t* n_frozen_queries) {
+    return draft_impl((Table*)h, (const Frozen*)hf, s, seq_len, T, crt, max_depth, tok, par, dep, mask, query_log, n_queries,
+                      frozen_log, n_frozen_queries);
 }
 
 // Ancestor-or-self mask of a given tree (parents precede children).

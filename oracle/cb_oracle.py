@@ -43,6 +43,12 @@ def lib():
         L.orc_table_dump.argtypes = [C.c_void_p] * 4
         L.orc_draft_tree.restype = C.c_int
         L.orc_draft_tree.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int] + [C.c_void_p] * 6
+        L.orc_frozen_new.restype = C.c_void_p
+        L.orc_frozen_new.argtypes = [C.c_int, C.c_int]
+        L.orc_frozen_free.argtypes = [C.c_void_p]
+        L.orc_frozen_add.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
+        L.orc_draft_tree_dual.restype = C.c_int
+        L.orc_draft_tree_dual.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int] + [C.c_void_p] * 8
         L.orc_tree_mask.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
         L.orc_argmax_f32.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_void_p]
         L.orc_accept.restype = C.c_int
@@ -131,6 +137,71 @@ class OracleTable:
         if with_log:
             return n, tok, par, dep, mask, [(tuple(int(x) for x in r[:-1]), int(r[-1])) for r in log[: nq.value]]
         return n, tok, par, dep, mask
+
+
+def frozen_build(corpus, LL, FL, LC, FC):
+    """Offline construction of the frozen table (paper Section 4.1, experimental set-up): the LC most frequent n-grams of
+    length LL become the leaders; each leader keeps the FC most frequent n-grams of length FL that follow it.
+
+    readings: the corpus is one token stream; an occurrence counts where LL + FL tokens are available, so every leader
+    has at least one follower; equal counts are ordered by the tokens, lexicographically smallest first.
+    Returns (leaders int32 [n, LL], n_followers int32 [n], followers int32 [n, FC, FL], -1 in unused places), leaders by
+    falling count, each leader's followers by falling count."""
+    from collections import Counter
+    c = [int(x) for x in np.asarray(corpus).reshape(-1)]
+    lead = Counter()
+    foll = {}
+    for i in range(len(c) - LL - FL + 1):
+        lk = tuple(c[i:i + LL])
+        lead[lk] += 1
+        foll.setdefault(lk, Counter())[tuple(c[i + LL:i + LL + FL])] += 1
+    top = sorted(lead.items(), key=lambda kv: (-kv[1], kv[0]))[:LC]
+    n = len(top)
+    leaders = np.full((n, LL), -1, np.int32)
+    nfol = np.zeros(n, np.int32)
+    followers = np.full((n, FC, FL), -1, np.int32)
+    for r, (lk, _) in enumerate(top):
+        leaders[r] = lk
+        fs = sorted(foll[lk].items(), key=lambda kv: (-kv[1], kv[0]))[:FC]
+        nfol[r] = len(fs)
+        for k, (fk, _) in enumerate(fs):
+            followers[r, k] = fk
+    return leaders, nfol, followers
+
+
+class OracleFrozen:
+    """Read-only table of Section 3.3, filled from frozen_build's arrays (or any arrays of that shape)."""
+
+    def __init__(self, LL, FL, leaders, n_followers, followers):
+        self.LL, self.FL = LL, FL
+        self._h = lib().orc_frozen_new(LL, FL)
+        leaders, n_followers, followers = _i32(leaders), _i32(n_followers), _i32(followers)
+        for r in range(leaders.shape[0]):
+            lib().orc_frozen_add(self._h, _p(leaders[r]), int(n_followers[r]), _p(np.ascontiguousarray(followers[r])))
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            lib().orc_frozen_free(self._h)
+            self._h = None
+
+
+def draft_tree_dual(table, frozen, tokens, seq_len, T, crt, max_depth, with_log=False):
+    """Dual-table draft (Section 3.3): `table` (OracleTable) forms the tree, `frozen` (OracleFrozen or None) grows it on."""
+    s = _i32(tokens)
+    W = (T + 31) // 32
+    tok = np.empty(T, dtype=np.int32)
+    par = np.empty(T, dtype=np.int32)
+    dep = np.empty(T, dtype=np.int32)
+    mask = np.empty((T, W), dtype=np.uint32)
+    log = np.full((max(T, 1) * 2, table.LL + 1), -1, dtype=np.int32)
+    flog = np.full((max(T, 1) * 2, table.LL + 1), -1, dtype=np.int32)
+    nq, nfq = C.c_int32(0), C.c_int32(0)
+    n = lib().orc_draft_tree_dual(table._h, frozen._h if frozen is not None else None, _p(s), int(seq_len), T, crt, max_depth,
+                                  _p(tok), _p(par), _p(dep), _p(mask), _p(log), C.addressof(nq), _p(flog), C.addressof(nfq))
+    if with_log:
+        unpack = lambda a, k: [(tuple(int(x) for x in r[:-1]), int(r[-1])) for r in a[:k]]
+        return n, tok, par, dep, mask, unpack(log, nq.value), unpack(flog, nfq.value)
+    return n, tok, par, dep, mask
 
 
 def tree_mask(par, n, T):
