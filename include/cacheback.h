@@ -221,6 +221,42 @@ typedef struct {
 cb_status cb_kv_commit(cb_ctx* ctx, const cb_kv_commit_args* args, void* stream);
 
 /*
+ * Frozen table (Section 3.3: besides the dynamic table, a second table is prepared offline from frequent
+ * leader-follower pairs of a large corpus; a decoding step first queries the dynamic table to form the draft tree and
+ * then the frozen one to grow the tree further while the size cap allows; the frozen table ignores insertions).
+ *
+ * A frozen table is one device buffer owned by the caller, of cb_frozen_bytes() bytes, 256-byte aligned, shared by every
+ * sequence and every context that attaches it, and only read by the step calls.  LL and FL must equal the context's;
+ * LC (1..2^20) and FC (1..16) are its own.
+ *
+ *   cb_frozen_load    fills the buffer from HOST arrays: leaders int32 [n_leaders, LL], n_followers int32 [n_leaders]
+ *                     (1..FC each), followers int32 [n_leaders, FC, FL], each leader's followers most frequent first,
+ *                     leaders most frequent first.  Synchronises the device.
+ *   cb_frozen_dump    the reverse, into HOST arrays sized for LC leaders (any may be NULL; unused follower places -1):
+ *                     leaders by falling corpus count, equal counts by rising tokens.  Synchronises the device.
+ *   cb_frozen_attach  makes cb_draft_tree of this context run the second pass; dev_table = NULL detaches.  Host call, no
+ *                     device work; order it against draft calls in flight yourself.
+ *
+ * With a frozen table attached, cb_draft_tree continues after the dynamic pass while the tree has fewer than max_nodes
+ * nodes: it visits, first in first out, every node that can carry a follower list (the root and the last node of every
+ * complete follower, in creation order; the ends of the complete followers the frozen pass adds join the queue), looks
+ * the node's key up in the frozen table and attaches the stored followers, most frequent first, under the same rules as
+ * the dynamic pass (a query at the root only while fewer than max(1, max_nodes - crt) nodes exist, any other while fewer
+ * than max_nodes; max_depth; a follower that does not fit is cut short).  Frozen followers are not compared with the
+ * branches already present.  Frozen queries touch no recency and are counted in CB_CNT_FROZEN_QUERIES / _HITS.
+ */
+typedef struct {
+    int32_t LL, FL, LC, FC;
+} cb_frozen_config;
+
+cb_status cb_frozen_bytes(const cb_frozen_config* cfg, size_t* bytes);
+cb_status cb_frozen_load(const cb_frozen_config* cfg, void* dev_table, size_t bytes, int32_t n_leaders,
+                         const int32_t* leaders, const int32_t* n_followers, const int32_t* followers);
+cb_status cb_frozen_dump(const cb_frozen_config* cfg, const void* dev_table, size_t bytes, int32_t* n_leaders,
+                         int32_t* leaders, int32_t* n_followers, int32_t* followers);
+cb_status cb_frozen_attach(cb_ctx* ctx, const cb_frozen_config* cfg, const void* dev_table, size_t bytes);
+
+/*
  * cb_accept_static — cb_accept (logits form) for callers that must not allocate device memory.
  * (The paper has no counterpart; this is a packaging variant of the call above.)
  *
@@ -277,6 +313,8 @@ enum {
     CB_CNT_QUERIES = 3,
     CB_CNT_QUERY_HITS = 4,
     CB_CNT_MAX_PROBE = 5,
+    CB_CNT_FROZEN_QUERIES = 6,
+    CB_CNT_FROZEN_HITS = 7,
     CB_NUM_COUNTERS = 8
 };
 cb_status cb_poll_status(cb_ctx* ctx, cb_status* device_status, uint64_t* counters);

@@ -1,5 +1,5 @@
 """Cacheback draft-and-verify step for NVIDIA B200 (sm_100a): C-ABI CUDA library + thin binding."""
-from .api import Cacheback, CachebackError, cb_accept_static
+from .api import Cacheback, CachebackError, FrozenTable, cb_accept_static
 from . import _lib
 
-__all__ = ["Cacheback", "CachebackError", "cb_accept_static", "_lib"]
+__all__ = ["Cacheback", "CachebackError", "FrozenTable", "cb_accept_static", "_lib"]

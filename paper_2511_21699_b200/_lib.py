@@ -13,16 +13,22 @@ CB_ERR_STATIC_LIMIT = 7
 CB_ERR_KV_FULL = 8
 CB_STATIC_MAX_BATCH, CB_STATIC_MAX_ROWS = 1024, 8192
 CB_NUM_COUNTERS = 8
-COUNTER_NAMES = ["inserts", "leader_evictions", "follower_evictions", "queries", "query_hits", "max_probe"]
+COUNTER_NAMES = ["inserts", "leader_evictions", "follower_evictions", "queries", "query_hits", "max_probe", "frozen_queries",
+                 "frozen_hits"]
 
 EXPORTS = ["cb_workspace_bytes", "cb_create", "cb_destroy", "cb_reset", "cb_update", "cb_draft_tree",
            "cb_tree_attn", "cb_accept", "cb_table_dump", "cb_table_load", "cb_poll_status", "cb_launch_count",
-           "cb_status_str", "cb_accept_static", "cb_kv_commit"]
+           "cb_status_str", "cb_accept_static", "cb_kv_commit", "cb_frozen_bytes", "cb_frozen_load", "cb_frozen_dump",
+           "cb_frozen_attach"]
 
 
 class CbConfigC(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("batch", "LL", "FL", "LC", "FC", "max_nodes", "crt", "max_depth", "vocab",
                                           "n_q_heads", "n_kv_heads", "head_dim", "page_size")] + [("flags", C.c_uint32)]
+
+
+class CbFrozenConfigC(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("LL", "FL", "LC", "FC")]
 
 
 class CbKvCommitArgsC(C.Structure):
@@ -62,6 +68,10 @@ def load():
     L.cb_table_dump.argtypes = [vp, i32, C.POINTER(i32), vp, vp, vp]
     L.cb_table_load.argtypes = [vp, i32, i32, vp, vp, vp]
     L.cb_poll_status.argtypes = [vp, C.POINTER(i32), vp]
+    L.cb_frozen_bytes.argtypes = [C.POINTER(CbFrozenConfigC), C.POINTER(C.c_size_t)]
+    L.cb_frozen_load.argtypes = [C.POINTER(CbFrozenConfigC), vp, C.c_size_t, i32, vp, vp, vp]
+    L.cb_frozen_dump.argtypes = [C.POINTER(CbFrozenConfigC), vp, C.c_size_t, C.POINTER(i32), vp, vp, vp]
+    L.cb_frozen_attach.argtypes = [vp, C.POINTER(CbFrozenConfigC), vp, C.c_size_t]
     L.cb_launch_count.restype = C.c_uint64
     L.cb_launch_count.argtypes = []
     L.cb_status_str.restype = C.c_char_p

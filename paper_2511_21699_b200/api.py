@@ -9,7 +9,7 @@ import numpy as np
 import torch
 
 from . import _lib
-from ._lib import CbConfigC, CbAttnArgsC, CbKvCommitArgsC
+from ._lib import CbConfigC, CbAttnArgsC, CbKvCommitArgsC, CbFrozenConfigC
 
 
 class CachebackError(RuntimeError):
@@ -63,6 +63,48 @@ def cb_accept_static(tree, logits, max_depth, res=None, stream=None):
                                 _ptr(res["out_tokens"], torch.int32), _ptr(res["target_ids"], torch.int32), _stream(stream)),
            "cb_accept_static")
     return res
+
+
+class FrozenTable:
+    """A frozen table (cb_frozen_*): one device buffer, owned by this object, that contexts attach read-only."""
+
+    def __init__(self, LL, FL, LC, FC, device="cuda:0"):
+        self.lib = _lib.load()
+        if not torch.cuda.is_available():
+            raise CachebackError("no CUDA device: the library has no CPU path")
+        self.device = torch.device(device)
+        self.cfg = CbFrozenConfigC(LL, FL, LC, FC)
+        nbytes = C.c_size_t(0)
+        _check(self.lib.cb_frozen_bytes(C.byref(self.cfg), C.byref(nbytes)), "cb_frozen_bytes")
+        self.bytes = nbytes.value
+        with torch.cuda.device(self.device):
+            self.buffer = torch.zeros(nbytes.value + 256, dtype=torch.uint8, device=self.device)
+        self.ptr = (self.buffer.data_ptr() + 255) // 256 * 256
+
+    def cb_frozen_load(self, leaders, n_followers, followers):
+        """Host arrays: leaders [n, LL], n_followers [n], followers [n, FC, FL], most frequent first."""
+        c = self.cfg
+        leaders = np.ascontiguousarray(leaders, dtype=np.int32).reshape(-1, c.LL)
+        n = leaders.shape[0]
+        nfol = np.ascontiguousarray(n_followers, dtype=np.int32).reshape(n)
+        fol = np.full((max(n, 1), c.FC, c.FL), -1, dtype=np.int32)
+        src = np.asarray(followers, dtype=np.int32).reshape(n, -1, c.FL)
+        fol[:n, : src.shape[1]] = src[:, : c.FC]
+        with torch.cuda.device(self.device):
+            _check(self.lib.cb_frozen_load(C.byref(self.cfg), self.ptr, self.bytes, n, leaders.ctypes.data, nfol.ctypes.data,
+                                           fol.ctypes.data), "cb_frozen_load")
+
+    def cb_frozen_dump(self):
+        """(leaders [n, LL], n_followers [n], followers [n, FC, FL]) as host arrays, most frequent first."""
+        c = self.cfg
+        n = C.c_int32(0)
+        leaders = np.empty((c.LC, c.LL), dtype=np.int32)
+        nfol = np.empty(c.LC, dtype=np.int32)
+        fol = np.empty((c.LC, c.FC, c.FL), dtype=np.int32)
+        with torch.cuda.device(self.device):
+            _check(self.lib.cb_frozen_dump(C.byref(self.cfg), self.ptr, self.bytes, C.byref(n), leaders.ctypes.data,
+                                           nfol.ctypes.data, fol.ctypes.data), "cb_frozen_dump")
+        return leaders[: n.value], nfol[: n.value], fol[: n.value]
 
 
 class Cacheback:
@@ -172,6 +214,14 @@ class Cacheback:
         return res
 
     # ---- helpers ------------------------------------------------------------------------------------
+    def cb_frozen_attach(self, frozen):
+        """frozen: a FrozenTable (kept alive by this object) or None to detach."""
+        if frozen is None:
+            _check(self.lib.cb_frozen_attach(self._h, None, None, 0), "cb_frozen_attach")
+        else:
+            _check(self.lib.cb_frozen_attach(self._h, C.byref(frozen.cfg), frozen.ptr, frozen.bytes), "cb_frozen_attach")
+        self._frozen = frozen
+
     def cb_table_dump(self, seq):
         """[(leader tuple, [follower tuples])], least recently used first (host lists)."""
         c = self.cfg

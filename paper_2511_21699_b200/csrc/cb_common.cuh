@@ -69,6 +69,8 @@ struct cb_ctx {
     char* ws;
     size_t ws_bytes;
     CbTables tables;
+    CbTables frozen;        // the read-only table of cb_frozen_attach (one "sequence", shared by the batch)
+    bool has_frozen;
     uint32_t* d_status;     // [4]
     unsigned long long* d_counters;  // [CB_NUM_COUNTERS]
     unsigned long long* d_rowmax;    // [batch * max_nodes] packed (value, index) maxima, zero between calls
@@ -87,6 +89,15 @@ struct CbLayout {
 };
 
 cb_status cb_compute_layout(const cb_config* cfg, CbLayout* L);
+
+// Device image of a frozen table: the single-sequence form of the layout above, in a buffer of its own.  lstamp holds each
+// leader's corpus count; a follower's stamp is FC - its rank by count, so the larger stamp is the more frequent follower.
+struct CbFrozenLayout {
+    uint32_t nslots, E;
+    size_t off_hdr, off_index, off_lstamp, off_entries, total;
+};
+cb_status cb_frozen_layout(const cb_frozen_config* cfg, CbFrozenLayout* L);
+CbTables cb_frozen_view(const cb_frozen_config* cfg, const CbFrozenLayout& L, void* dev_table);
 void cb_count_launch(int n);
 
 #define CB_ATTN_MAX_UNITS 640   // partial row tiles (128 rows x (D + 4) floats): 2 shared units x 2 row tiles per persistent CTA, 160 CTAs

@@ -181,14 +181,17 @@ __global__ void __launch_bounds__(128) cb_update_kernel(CbTables t, int B, const
 // the staged results, which fixes node indices, the point where the size cap ends the level and the
 // ordinal of every query that the sequential order would have issued; (3) the leaders of those queries
 // get their new recency stamp with an atomic max (two leaves of one level may share a leader).
+// With a frozen table attached (Section 3.3) a second pass follows while the tree is below the size cap: its first
+// frontier is every node that was a frontier leaf of the first pass, in creation order, and its lookups go to the
+// frozen table, which is shared by all sequences and only read (no clock tick, no stamp).
 struct DraftSmem {
     int32_t* tok; int32_t* par; int32_t* dep;
-    int32_t* front; int32_t* next;
+    int32_t* front; int32_t* next; int32_t* pts;
     int32_t* r_eid; int32_t* r_nf; int32_t* r_ok; uint32_t* r_stamp;
     int32_t* fol;
 };
 
-__global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, int T, int crt, int max_depth, int NL,
+__global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, int T, int crt, int max_depth, int NL, int FCmax,
                                                        const int32_t* __restrict__ tokens, int64_t row_stride,
                                                        const int32_t* __restrict__ seq_len,
                                                        int32_t* __restrict__ o_tok, int32_t* __restrict__ o_par,
@@ -199,109 +202,130 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, int T, int cr
     extern __shared__ int32_t smem[];
     DraftSmem S;
     S.tok = smem; S.par = S.tok + T; S.dep = S.par + T;
-    S.front = S.dep + T; S.next = S.front + NL;
-    S.r_eid = S.next + NL; S.r_nf = S.r_eid + NL; S.r_ok = S.r_nf + NL; S.r_stamp = (uint32_t*)(S.r_ok + NL);
+    S.front = S.dep + T; S.next = S.front + NL; S.pts = S.next + NL;
+    S.r_eid = S.pts + NL; S.r_nf = S.r_eid + NL; S.r_ok = S.r_nf + NL; S.r_stamp = (uint32_t*)(S.r_ok + NL);
     S.fol = (int32_t*)(S.r_stamp + NL);
-    __shared__ int sh_n, sh_nfront, sh_nnext, sh_q, sh_hits, sh_level;
+    __shared__ int sh_n, sh_nfront, sh_nnext, sh_npts, sh_q, sh_hits, sh_fq, sh_fhits;
 
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     const CbSeq s = cb_seq(t, b);
     const int32_t* row = tokens + (size_t)b * row_stride;
     const int L = seq_len[b];
     const int W = (T + 31) >> 5;
-    const int FLFC = t.FL * t.FC;
+    const int FLFC = t.FL * FCmax;
     const uint32_t clock0 = s.hdr[0];
+    const bool has_frozen = tf.index != nullptr;
 
     for (int i = tid; i < T; i += blockDim.x) { S.tok[i] = -1; S.par[i] = -1; S.dep[i] = -1; }
     if (tid == 0) {
-        sh_n = 0; sh_nfront = 0; sh_q = 0; sh_hits = 0; sh_level = 1;
+        sh_n = 0; sh_nfront = 0; sh_npts = 0; sh_q = 0; sh_hits = 0; sh_fq = 0; sh_fhits = 0;
     }
     __syncthreads();
     if (tid == 0 && L >= 1) {
-        S.tok[0] = row[L - 1]; S.dep[0] = 0; sh_n = 1; S.front[0] = 0; sh_nfront = 1;
+        S.tok[0] = row[L - 1]; S.dep[0] = 0; sh_n = 1; S.front[0] = 0; sh_nfront = 1; S.pts[0] = 0; sh_npts = 1;
     }
     __syncthreads();
 
-    while (true) {
-        const int nfront = sh_nfront, n_now = sh_n;
-        if (nfront == 0 || n_now >= T) break;
-        // (1) parallel lookups, one warp per leaf
-        for (int li = warp; li < nfront; li += nwarps) {
-            const int leaf = S.front[li];
-            const int d = S.dep[leaf];
-            // key = last LL tokens of (row[0 .. L-1) ++ root->leaf path); lane j < LL holds key[j]
-            int32_t mykey = 0;
-            bool ok = d < max_depth;
-            if (lane < t.LL) {
-                const int back = t.LL - 1 - lane;         // distance from the leaf along the sequence
-                if (back <= d) {
-                    int c = leaf;
-                    for (int k = 0; k < back; ++k) c = S.par[c];
-                    mykey = S.tok[c];
-                } else {
-                    const int pos = L - 1 - (back - d);
-                    mykey = pos >= 0 ? row[pos] : -1;
-                }
-            }
-            ok = ok && __all_sync(CB_FULL, mykey >= 0);
-            int eid = -1, nf = 0;
-            if (ok) {
-                const uint64_t h = warp_hash(t, mykey);
-                const Probe pr = tbl_find(t, s, mykey, h, lane);
-                if (pr.eid == -2 && lane == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_PROBE_LIMIT);
-                if (pr.eid >= 0) {
-                    eid = pr.eid;
-                    const uint32_t* e = s.entries + (size_t)eid * t.E;
-                    const uint32_t fs = lane < t.FC ? e[t.LL + lane] : 0u;
-                    // rank = number of followers inserted more recently than mine (stamps are unique)
-                    int rank = 0;
-                    for (int f = 0; f < t.FC; ++f) {
-                        const uint32_t o = __shfl_sync(CB_FULL, fs, f);
-                        rank += (o > fs) ? 1 : 0;
-                    }
-                    nf = __popc(__ballot_sync(CB_FULL, fs != 0u));
-                    if (lane < t.FC && fs != 0u)
-                        for (int j = 0; j < t.FL; ++j)
-                            S.fol[li * FLFC + rank * t.FL + j] = (int32_t)e[t.LL + t.FC + lane * t.FL + j];
-                }
-            }
-            if (lane == 0) { S.r_eid[li] = eid; S.r_nf[li] = nf; S.r_ok[li] = ok ? 1 : 0; S.r_stamp[li] = 0u; }
+    for (int pass = 0; pass < (has_frozen ? 2 : 1); ++pass) {
+        const CbTables& tt = pass ? tf : t;
+        const CbSeq ss = pass ? cb_seq(tf, 0) : s;
+        if (pass == 1) {
+            // the frozen pass starts from every frontier leaf the dynamic pass had
+            const int np = sh_npts;
+            __syncthreads();
+            for (int i = tid; i < np; i += blockDim.x) S.front[i] = S.pts[i];
+            if (tid == 0) sh_nfront = np;
+            __syncthreads();
         }
-        __syncthreads();
-        // (2) sequential replay of the breadth-first order
-        if (tid == 0) {
-            int n = n_now, q = sh_q, hits = sh_hits, nn = 0;
-            const int cap = (sh_level == 1) ? max(1, T - crt) : T;
-            for (int li = 0; li < nfront; ++li) {
-                if (n >= cap) break;
-                if (!S.r_ok[li]) continue;
-                ++q;                                            // this query is issued: the clock ticks
-                if (S.r_eid[li] < 0) continue;
-                ++hits;
-                S.r_stamp[li] = clock0 + (uint32_t)q;
+        while (true) {
+            const int nfront = sh_nfront, n_now = sh_n;
+            if (nfront == 0 || n_now >= T) break;
+            // (1) parallel lookups, one warp per leaf
+            for (int li = warp; li < nfront; li += nwarps) {
                 const int leaf = S.front[li];
-                for (int f = 0; f < S.r_nf[li]; ++f) {
-                    if (n >= cap) break;
-                    int p = leaf, k = 0;
-                    for (int j = 0; j < t.FL; ++j) {
-                        if (n >= cap || S.dep[p] >= max_depth) break;
-                        S.tok[n] = S.fol[li * FLFC + f * t.FL + j];
-                        S.par[n] = p; S.dep[n] = S.dep[p] + 1; p = n; ++n; ++k;
+                const int d = S.dep[leaf];
+                // key = last LL tokens of (row[0 .. L-1) ++ root->leaf path); lane j < LL holds key[j]
+                int32_t mykey = 0;
+                bool ok = d < max_depth;
+                if (lane < t.LL) {
+                    const int back = t.LL - 1 - lane;         // distance from the leaf along the sequence
+                    if (back <= d) {
+                        int c = leaf;
+                        for (int k = 0; k < back; ++k) c = S.par[c];
+                        mykey = S.tok[c];
+                    } else {
+                        const int pos = L - 1 - (back - d);
+                        mykey = pos >= 0 ? row[pos] : -1;
                     }
-                    if (k == t.FL) S.next[nn++] = p;
                 }
+                ok = ok && __all_sync(CB_FULL, mykey >= 0);
+                int eid = -1, nf = 0;
+                if (ok) {
+                    const uint64_t h = warp_hash(tt, mykey);
+                    const Probe pr = tbl_find(tt, ss, mykey, h, lane);
+                    if (pr.eid == -2 && lane == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_PROBE_LIMIT);
+                    if (pr.eid >= 0) {
+                        eid = pr.eid;
+                        const uint32_t* e = ss.entries + (size_t)eid * tt.E;
+                        const uint32_t fs = lane < tt.FC ? e[tt.LL + lane] : 0u;
+                        // rank = number of followers with a larger stamp than mine (stamps are unique): more recently
+                        // inserted in the dynamic table, more frequent in the frozen one
+                        int rank = 0;
+                        for (int f = 0; f < tt.FC; ++f) {
+                            const uint32_t o = __shfl_sync(CB_FULL, fs, f);
+                            rank += (o > fs) ? 1 : 0;
+                        }
+                        nf = __popc(__ballot_sync(CB_FULL, fs != 0u));
+                        if (lane < tt.FC && fs != 0u)
+                            for (int j = 0; j < tt.FL; ++j)
+                                S.fol[li * FLFC + rank * tt.FL + j] = (int32_t)e[tt.LL + tt.FC + lane * tt.FL + j];
+                    }
+                }
+                if (lane == 0) { S.r_eid[li] = eid; S.r_nf[li] = nf; S.r_ok[li] = ok ? 1 : 0; S.r_stamp[li] = 0u; }
             }
-            sh_n = n; sh_q = q; sh_hits = hits; sh_nnext = nn; sh_level = sh_level + 1;
+            __syncthreads();
+            // (2) sequential replay of the breadth-first order.  A query at the root (the only leaf of level 1) is issued,
+            // and its followers attached, while the tree has fewer than max(1, T - crt) nodes; any other while fewer than T.
+            if (tid == 0) {
+                int n = n_now, q = 0, hits = 0, nn = 0;
+                for (int li = 0; li < nfront; ++li) {
+                    if (n >= T) break;
+                    const int leaf = S.front[li];
+                    const int cap = leaf == 0 ? max(1, T - crt) : T;
+                    if (n >= cap) continue;
+                    if (!S.r_ok[li]) continue;
+                    ++q;                                        // this query is issued: the dynamic table's clock ticks
+                    if (S.r_eid[li] < 0) continue;
+                    ++hits;
+                    if (pass == 0) S.r_stamp[li] = clock0 + (uint32_t)(sh_q + q);
+                    for (int f = 0; f < S.r_nf[li]; ++f) {
+                        if (n >= cap) break;
+                        int p = leaf, k = 0;
+                        for (int j = 0; j < t.FL; ++j) {
+                            if (n >= cap || S.dep[p] >= max_depth) break;
+                            S.tok[n] = S.fol[li * FLFC + f * t.FL + j];
+                            S.par[n] = p; S.dep[n] = S.dep[p] + 1; p = n; ++n; ++k;
+                        }
+                        if (k == t.FL) S.next[nn++] = p;
+                    }
+                }
+                sh_n = n; sh_nnext = nn;
+                if (pass == 0) { sh_q += q; sh_hits += hits; } else { sh_fq += q; sh_fhits += hits; }
+            }
+            __syncthreads();
+            // (3) stamp the leaders the sequential order reached; publish the next frontier
+            if (pass == 0)
+                for (int li = tid; li < nfront; li += blockDim.x)
+                    if (S.r_stamp[li] != 0u) atomicMax(&s.lstamp[S.r_eid[li]], S.r_stamp[li]);
+            const int nn = sh_nnext, np = sh_npts;
+            __syncthreads();
+            for (int i = tid; i < nn; i += blockDim.x) {
+                S.front[i] = S.next[i];
+                if (pass == 0 && has_frozen) S.pts[np + i] = S.next[i];
+            }
+            if (tid == 0) { sh_nfront = nn; if (pass == 0 && has_frozen) sh_npts = np + nn; }
+            __syncthreads();
         }
-        __syncthreads();
-        // (3) stamp the leaders the sequential order reached; publish the next frontier
-        for (int li = tid; li < nfront; li += blockDim.x)
-            if (S.r_stamp[li] != 0u) atomicMax(&s.lstamp[S.r_eid[li]], S.r_stamp[li]);
-        const int nn = sh_nnext;
-        __syncthreads();
-        for (int i = tid; i < nn; i += blockDim.x) S.front[i] = S.next[i];
-        if (tid == 0) sh_nfront = nn;
-        __syncthreads();
     }
 
     const int n = sh_n;
@@ -310,6 +334,8 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, int T, int cr
         o_n[b] = n;
         if (sh_q) atomicAdd(&counters[CB_CNT_QUERIES], (unsigned long long)sh_q);
         if (sh_hits) atomicAdd(&counters[CB_CNT_QUERY_HITS], (unsigned long long)sh_hits);
+        if (sh_fq) atomicAdd(&counters[CB_CNT_FROZEN_QUERIES], (unsigned long long)sh_fq);
+        if (sh_fhits) atomicAdd(&counters[CB_CNT_FROZEN_HITS], (unsigned long long)sh_fhits);
     }
     for (int i = tid; i < T; i += blockDim.x) {
         o_tok[(size_t)b * T + i] = S.tok[i];
@@ -341,11 +367,14 @@ extern "C" cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t r
     const cb_config& c = ctx->cfg;
     const int T = c.max_nodes;
     const int NL = min(T, (T - 1) / c.FL + 1);
-    const size_t smem = sizeof(int32_t) * ((size_t)3 * T + (size_t)6 * NL + (size_t)NL * c.FL * c.FC);
+    const int FCmax = ctx->has_frozen ? max(c.FC, ctx->frozen.FC) : c.FC;
+    const size_t smem = sizeof(int32_t) * ((size_t)3 * T + (size_t)7 * NL + (size_t)NL * c.FL * FCmax);
     if (smem > 48 * 1024) return CB_ERR_UNSUPPORTED;
     const int threads = 32 * max(1, min(8, NL));
-    CB_CUDA(cb_launch_pdl(cb_draft_kernel, dim3(c.batch), dim3(threads), smem, (cudaStream_t)stream, ctx->tables, T, c.crt, c.max_depth, NL, tokens,
-                          row_stride, seq_len, tree_tokens, tree_parent, tree_depth, tree_mask, n_nodes, ctx->d_status, ctx->d_counters));
+    CbTables tf = {};
+    if (ctx->has_frozen) tf = ctx->frozen;
+    CB_CUDA(cb_launch_pdl(cb_draft_kernel, dim3(c.batch), dim3(threads), smem, (cudaStream_t)stream, ctx->tables, tf, T, c.crt, c.max_depth, NL, FCmax,
+                          tokens, row_stride, seq_len, tree_tokens, tree_parent, tree_depth, tree_mask, n_nodes, ctx->d_status, ctx->d_counters));
     cb_count_launch(1);
     return CB_OK;
 }
