@@ -244,6 +244,15 @@ cb_status cb_kv_commit(cb_ctx* ctx, const cb_kv_commit_args* args, void* stream)
  * the dynamic pass (a query at the root only while fewer than max(1, max_nodes - crt) nodes exist, any other while fewer
  * than max_nodes; max_depth; a follower that does not fit is cut short).  Frozen followers are not compared with the
  * branches already present.  Frozen queries touch no recency and are counted in CB_CNT_FROZEN_QUERIES / _HITS.
+ *
+ * Offline construction (Section 4.1: from a corpus sample, the LC most frequent n-grams of length LL become the leaders,
+ * and each leader keeps the FC most frequent n-grams of length FL that follow it).
+ *   cb_frozen_build   counts on the GPU.  dev_corpus int32 [n_tokens] (device, ids >= 0, one token stream,
+ *                     n_tokens <= 2^30); an occurrence is counted where LL + FL tokens are available, so every leader
+ *                     has at least one follower; equal counts are ordered by the tokens, smallest first.  dev_scratch:
+ *                     cb_frozen_build_bytes() bytes of device memory, 256-byte aligned, free again after the call.
+ *                     Overwrites dev_table.  Enqueues on `stream` and waits for it; returns CB_ERR_INVALID_ARG if a
+ *                     negative token was met (its windows are left out).
  */
 typedef struct {
     int32_t LL, FL, LC, FC;
@@ -255,6 +264,9 @@ cb_status cb_frozen_load(const cb_frozen_config* cfg, void* dev_table, size_t by
 cb_status cb_frozen_dump(const cb_frozen_config* cfg, const void* dev_table, size_t bytes, int32_t* n_leaders,
                          int32_t* leaders, int32_t* n_followers, int32_t* followers);
 cb_status cb_frozen_attach(cb_ctx* ctx, const cb_frozen_config* cfg, const void* dev_table, size_t bytes);
+cb_status cb_frozen_build_bytes(const cb_frozen_config* cfg, int64_t n_tokens, size_t* scratch_bytes);
+cb_status cb_frozen_build(const cb_frozen_config* cfg, const int32_t* dev_corpus, int64_t n_tokens, void* dev_table,
+                          size_t table_bytes, void* dev_scratch, size_t scratch_bytes, void* stream);
 
 /*
  * cb_accept_static — cb_accept (logits form) for callers that must not allocate device memory.

@@ -19,7 +19,7 @@ COUNTER_NAMES = ["inserts", "leader_evictions", "follower_evictions", "queries",
 EXPORTS = ["cb_workspace_bytes", "cb_create", "cb_destroy", "cb_reset", "cb_update", "cb_draft_tree",
            "cb_tree_attn", "cb_accept", "cb_table_dump", "cb_table_load", "cb_poll_status", "cb_launch_count",
            "cb_status_str", "cb_accept_static", "cb_kv_commit", "cb_frozen_bytes", "cb_frozen_load", "cb_frozen_dump",
-           "cb_frozen_attach"]
+           "cb_frozen_attach", "cb_frozen_build_bytes", "cb_frozen_build"]
 
 
 class CbConfigC(C.Structure):
@@ -72,6 +72,8 @@ def load():
     L.cb_frozen_load.argtypes = [C.POINTER(CbFrozenConfigC), vp, C.c_size_t, i32, vp, vp, vp]
     L.cb_frozen_dump.argtypes = [C.POINTER(CbFrozenConfigC), vp, C.c_size_t, C.POINTER(i32), vp, vp, vp]
     L.cb_frozen_attach.argtypes = [vp, C.POINTER(CbFrozenConfigC), vp, C.c_size_t]
+    L.cb_frozen_build_bytes.argtypes = [C.POINTER(CbFrozenConfigC), i64, C.POINTER(C.c_size_t)]
+    L.cb_frozen_build.argtypes = [C.POINTER(CbFrozenConfigC), vp, i64, vp, C.c_size_t, vp, C.c_size_t, vp]
     L.cb_launch_count.restype = C.c_uint64
     L.cb_launch_count.argtypes = []
     L.cb_status_str.restype = C.c_char_p

@@ -94,6 +94,19 @@ class FrozenTable:
             _check(self.lib.cb_frozen_load(C.byref(self.cfg), self.ptr, self.bytes, n, leaders.ctypes.data, nfol.ctypes.data,
                                            fol.ctypes.data), "cb_frozen_load")
 
+    def cb_frozen_build(self, corpus, stream=None):
+        """corpus: int32 CUDA tensor [n_tokens].  Counts on the GPU and overwrites this table; the scratch is a temporary
+        torch tensor."""
+        n = int(corpus.numel())
+        nbytes = C.c_size_t(0)
+        _check(self.lib.cb_frozen_build_bytes(C.byref(self.cfg), n, C.byref(nbytes)), "cb_frozen_build_bytes")
+        with torch.cuda.device(self.device):
+            scratch = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
+            sp = (scratch.data_ptr() + 255) // 256 * 256
+            _check(self.lib.cb_frozen_build(C.byref(self.cfg), _ptr(corpus, torch.int32), n, self.ptr, self.bytes, sp, nbytes.value,
+                                            _stream(stream)), "cb_frozen_build")
+        del scratch
+
     def cb_frozen_dump(self):
         """(leaders [n, LL], n_followers [n], followers [n, FC, FL]) as host arrays, most frequent first."""
         c = self.cfg

@@ -136,3 +136,61 @@ def test_only_frozen(oracle):
         assert cb.cb_table_dump(0) == []
     assert max(sizes) > 1
     assert cb.cb_poll_status()[0] == 0
+
+
+# ------------------------------------------------------------------------------------------------ builder on the GPU
+def _build_and_compare(oracle, corpus, LL, FL, LC, FC):
+    from paper_2511_21699_b200 import FrozenTable
+    ft = FrozenTable(LL, FL, LC, FC)
+    ft.cb_frozen_build(dev(np.asarray(corpus, np.int32)))
+    L, nf, F = ft.cb_frozen_dump()
+    oL, onf, oF = oracle.frozen_build(corpus, LL, FL, LC, FC)
+    assert L.shape == oL.shape, (L.shape, oL.shape)
+    assert np.array_equal(L, oL) and np.array_equal(nf, onf) and np.array_equal(F, oF)
+    return ft, len(L)
+
+
+@pytest.mark.parametrize("LL,FL,LC,FC,vocab,n", [(1, 3, 64, 4, 300, 20000),      # more distinct leaders than LC
+                                                 (1, 3, 1024, 16, 300, 20000),   # all leaders fit; FC at its maximum
+                                                 (2, 2, 500, 3, 12, 30000),      # tiny vocabulary: many equal counts
+                                                 (3, 1, 777, 5, 6, 9000),
+                                                 (4, 8, 2048, 2, 40, 15000),     # longest leader and follower
+                                                 (2, 3, 16, 1, 1000, 5000)])     # nearly every count is 1: ties decide
+def test_builder_matches_the_oracle(oracle, LL, FL, LC, FC, vocab, n):
+    rng = np.random.default_rng(LL * 100 + FL)
+    corpus = (rng.zipf(1.3, n) % vocab).astype(np.int32)
+    _, got = _build_and_compare(oracle, corpus, LL, FL, LC, FC)
+    assert got > 0
+
+
+def test_builder_on_the_workload_corpus_and_reuse(oracle):
+    """The table the closed-loop tests load from the oracle's builder, built on the GPU instead; building twice into the
+    same buffers gives the same table."""
+    from paper_2511_21699_b200 import Cacheback
+    cfg = W.get_config("c2_7b")
+    corpus = _corpus(cfg, 60000)
+    ft, n = _build_and_compare(oracle, corpus, cfg.LL, cfg.FL, 4096, 6)
+    first = ft.cb_frozen_dump()
+    ft.cb_frozen_build(dev(corpus))
+    again = ft.cb_frozen_dump()
+    assert all(np.array_equal(a, b) for a, b in zip(first, again))
+    # the built table drives the draft like the loaded one
+    ofz = oracle.OracleFrozen(cfg.LL, cfg.FL, *first)
+    cb = Cacheback.from_config(cfg)
+    cb.cb_frozen_attach(ft)
+    prob = Problem(cfg)
+    pos = np.full(cfg.batch, 40, np.int32)
+    tree = cb.cb_draft_tree(dev(prob.toks), dev(pos))
+    for b in range(cfg.batch):
+        empty = oracle.OracleTable(cfg.LL, cfg.FL, cfg.LC, cfg.FC)
+        nn, tok, par, dep, mask = oracle.draft_tree_dual(empty, ofz, prob.toks[b], 40, cfg.max_nodes, cfg.crt, cfg.max_depth)
+        assert int(tree["n_nodes"][b]) == nn and np.array_equal(tree["tokens"][b].cpu().numpy(), tok)
+
+
+def test_builder_edge_cases(oracle):
+    from paper_2511_21699_b200 import FrozenTable, CachebackError
+    for corpus in ([], [5], [1, 2, 3], [1, 2, 3, 4], [7] * 50):
+        _build_and_compare(oracle, np.array(corpus, np.int32), 1, 3, 8, 2)
+    ft = FrozenTable(1, 2, 8, 2)
+    with pytest.raises(CachebackError):
+        ft.cb_frozen_build(dev(np.array([1, 2, -1, 3, 4, 5], np.int32)))     # negative ids are rejected
