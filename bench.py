@@ -35,6 +35,8 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--full-trees", action="store_true", help="attention/acceptance on synthetic full-size trees")
+    ap.add_argument("--frozen", type=int, default=0, metavar="TOKENS",
+                    help="attach a frozen table built on the GPU from a synthetic corpus of this many tokens (0 = none)")
     return ap.parse_args()
 
 
@@ -278,6 +280,22 @@ def run_ours(args, rank, world, local_rank):
     n_old = dev(np.stack([prefill + ADVANCE * s for s in range(total)]).astype(np.int32))
     n_new = dev(np.stack([prefill + ADVANCE * (s + 1) for s in range(total)]).astype(np.int32))
     cb.cb_update(toks_d, dev(np.zeros(B, np.int32)), dev(prefill))          # prompt initialisation, untimed
+    frozen_info = None
+    if args.frozen > 0:
+        # Stand-in for the paper's corpus sample: streams of the workload's own token distribution under other seeds.
+        from paper_2511_21699_b200 import FrozenTable
+        nseg = max(1, args.frozen // (1 << 20))
+        corpus = dev(np.concatenate([W.make_stream(cfg, 1000 + k, args.frozen // nseg) for k in range(nseg)]).astype(np.int32))
+        ft = FrozenTable(cfg.LL, cfg.FL, 1 << 16, min(16, 2 * cfg.FC), device=device)
+        ft.cb_frozen_build(corpus)                            # warm-up build
+        fe0, fe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fe0.record()
+        ft.cb_frozen_build(corpus)
+        fe1.record()
+        torch.cuda.synchronize()
+        cb.cb_frozen_attach(ft)
+        frozen_info = {"corpus_tokens": int(corpus.numel()), "LC": 1 << 16, "FC": min(16, 2 * cfg.FC),
+                       "leaders": int(len(ft.cb_frozen_dump()[0])), "build_ms": fe0.elapsed_time(fe1)}
     trees = [cb.alloc_tree() for _ in range(total)]         # every step keeps its own tree, so later passes can reuse it
     res = cb.alloc_accept()
     if args.full_trees:
@@ -442,7 +460,8 @@ def run_ours(args, rank, world, local_rank):
         "config": {"workload": cfg.name, "batch": B, "tree_cap": T, "mean_tree_nodes": float(nn_attn.mean()),
                    "context": [int(ctx.min()), int(ctx.max())], "l2": "rotating %d copies of K/V pool and logits (%.0f MB)" %
                    (R, R * (pool_bytes + logit_bytes) / 1e6), "launch": "CUDA graph of the timed steps, replayed %d times, median" % reps,
-                   "trees": "synthetic full" if args.full_trees else "drafted", "parallelism": "replicas x%d" % world},
+                   "trees": "synthetic full" if args.full_trees else "drafted", "frozen_table": frozen_info,
+                   "parallelism": "replicas x%d" % world},
         "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "ms_per_step": 1e3 * e2e_s / K},
