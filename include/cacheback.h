@@ -60,7 +60,7 @@ enum {
 /*
  * Shape of one context. Table parameters follow Section 3.1 / 3.2:
  *   LL, FL  leader / follower length in tokens          (1..4, 1..8)
- *   LC, FC  leader capacity per sequence, follower capacity per leader   (1..2^20, 1..16)
+ *   LC, FC  leader capacity per sequence, follower capacity per leader   (1..2^20, 1..128)
  *   max_nodes  tree-size cap, root included: the paper's total draft length (TDL)   (1..128)
  *   crt        nodes reserved for query levels >= 2: level 1 fills at most max(1, max_nodes - crt)
  *   max_depth  deepest node depth allowed (root = 0)
@@ -227,7 +227,7 @@ cb_status cb_kv_commit(cb_ctx* ctx, const cb_kv_commit_args* args, void* stream)
  *
  * A frozen table is one device buffer owned by the caller, of cb_frozen_bytes() bytes, 256-byte aligned, shared by every
  * sequence and every context that attaches it, and only read by the step calls.  LL and FL must equal the context's;
- * LC (1..2^20) and FC (1..16) are its own.
+ * LC (1..2^20) and FC (1..128) are its own.
  *
  *   cb_frozen_load    fills the buffer from HOST arrays: leaders int32 [n_leaders, LL], n_followers int32 [n_leaders]
  *                     (1..FC each), followers int32 [n_leaders, FC, FL], each leader's followers most frequent first,

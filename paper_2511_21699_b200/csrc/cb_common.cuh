@@ -15,7 +15,7 @@
 #define CB_MAX_T 128
 #define CB_MAX_LL 4
 #define CB_MAX_FL 8
-#define CB_MAX_FC 16
+#define CB_MAX_FC 128
 
 // Per-sequence table in the workspace (all 32-bit words):
 //   hdr[4]            clock, leader count, unused, unused

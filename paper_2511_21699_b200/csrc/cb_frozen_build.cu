@@ -8,9 +8,9 @@
 //   2. the LC best leaders under the order (count falling, tokens rising) are found by a most-significant-digit-first
 //      radix select over the distinct leaders (one histogram pass per byte of the composite key), then written into the
 //      frozen table's entries and hashed into its index;
-//   3. follower counts: windows whose leader was selected insert-or-increment the whole window in a second table, and
-//      every distinct window is pushed on its leader's list;
-//   4. every distinct window walks its leader's list and counts the windows that beat it under (count falling, follower
+//   3. follower counts: windows whose leader was selected insert-or-increment the whole window in a second table; the
+//      distinct windows are then grouped by leader into one array (count per leader, exclusive scan, scatter);
+//   4. every distinct window scans its leader's group and counts the windows that beat it under (count falling, follower
 //      tokens rising), giving up at FC; a rank below FC is that follower's place in the entry.
 // Which occurrence represents a key, and which entry id a leader gets, depends on timing; the table's content (and
 // cb_frozen_dump's output) does not.
@@ -35,8 +35,9 @@ struct BuildView {
     BuildState* st;
     uint32_t* h1_pos; uint32_t* h1_cnt; int32_t* h1_eid;          // [S] leaders
     uint32_t* uniq;                                               // [M] slots of the distinct leaders
-    uint32_t* h2_pos; uint32_t* h2_cnt; int32_t* h2_eid; uint32_t* h2_next;   // [S] windows of selected leaders
-    uint32_t* head;                                               // [LC] list heads per entry
+    uint32_t* h2_pos; uint32_t* h2_cnt; int32_t* h2_eid;          // [S] windows of selected leaders
+    uint32_t* seg; uint32_t* seg_cnt;                             // [S] distinct windows grouped by leader: slot, count
+    uint32_t* grp_n; uint32_t* grp_off; uint32_t* grp_fill;       // [LC] group size, start, scatter cursor per entry
     uint32_t S;                                                   // slots of each hash table (a power of two)
     const int32_t* corpus;
     uint32_t M;
@@ -84,9 +85,9 @@ __global__ void fb_init_kernel(BuildView v, CbTables t) {
     const size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (size_t)gridDim.x * blockDim.x;
     for (size_t i = g; i < v.S; i += stride) {
         v.h1_pos[i] = kEmpty; v.h1_cnt[i] = 0u; v.h1_eid[i] = -1;
-        v.h2_pos[i] = kEmpty; v.h2_cnt[i] = 0u; v.h2_eid[i] = -1; v.h2_next[i] = kEmpty;
+        v.h2_pos[i] = kEmpty; v.h2_cnt[i] = 0u; v.h2_eid[i] = -1;
     }
-    for (size_t i = g; i < (size_t)v.LC; i += stride) { v.head[i] = kEmpty; t.lstamp[i] = 0u; }
+    for (size_t i = g; i < (size_t)v.LC; i += stride) { v.grp_n[i] = 0u; v.grp_off[i] = 0u; v.grp_fill[i] = 0u; t.lstamp[i] = 0u; }
     for (size_t i = g; i < t.nslots; i += stride) t.index[i] = CB_IDX_EMPTY;
     for (size_t i = g; i < (size_t)v.LC * t.E; i += stride) t.entries[i] = 0u;
     if (g < sizeof(BuildState) / 4) reinterpret_cast<uint32_t*>(v.st)[g] = 0u;
@@ -190,7 +191,7 @@ __global__ void fb_place_leaders_kernel(BuildView v, CbTables t) {
     if (blockIdx.x == 0 && threadIdx.x == 0) t.hdr[1] = min(n, (uint32_t)v.LC);
 }
 
-// 3. follower counts of the selected leaders; distinct windows are linked to their leader
+// 3a. follower counts of the selected leaders; every leader learns how many distinct windows it has
 __global__ void fb_count_followers_kernel(BuildView v) {
     const size_t stride = (size_t)gridDim.x * blockDim.x;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < v.M; i += stride) {
@@ -207,8 +208,37 @@ __global__ void fb_count_followers_kernel(BuildView v) {
         atomicAdd(&v.h2_cnt[s], 1u);
         if (created) {
             v.h2_eid[s] = eid;
-            v.h2_next[s] = atomicExch(&v.head[eid], s);
+            atomicAdd(&v.grp_n[eid], 1u);
         }
+    }
+}
+// 3b. exclusive scan of the group sizes (one block; each thread owns a contiguous run of entries)
+__global__ void __launch_bounds__(1024) fb_group_scan_kernel(BuildView v) {
+    __shared__ uint32_t part[1024];
+    const uint32_t n = v.st->n_sel < (uint32_t)v.LC ? v.st->n_sel : (uint32_t)v.LC;
+    const uint32_t per = (n + 1023u) / 1024u, lo = threadIdx.x * per, hi = min(n, lo + per);
+    uint32_t sum = 0;
+    for (uint32_t i = lo; i < hi; ++i) sum += v.grp_n[i];
+    part[threadIdx.x] = sum;
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {
+        const uint32_t add = threadIdx.x >= o ? part[threadIdx.x - o] : 0u;
+        __syncthreads();
+        part[threadIdx.x] += add;
+        __syncthreads();
+    }
+    uint32_t run = part[threadIdx.x] - sum;
+    for (uint32_t i = lo; i < hi; ++i) { v.grp_off[i] = run; run += v.grp_n[i]; }
+}
+// 3c. the distinct windows, grouped by leader, with their counts beside them
+__global__ void fb_group_scatter_kernel(BuildView v) {
+    const size_t stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t s = (size_t)blockIdx.x * blockDim.x + threadIdx.x; s < v.S; s += stride) {
+        if (v.h2_pos[s] == kEmpty) continue;
+        const int32_t eid = v.h2_eid[s];
+        const uint32_t at = v.grp_off[eid] + atomicAdd(&v.grp_fill[eid], 1u);
+        v.seg[at] = (uint32_t)s;
+        v.seg_cnt[at] = v.h2_cnt[s];
     }
 }
 
@@ -220,13 +250,15 @@ __global__ void fb_rank_followers_kernel(BuildView v, CbTables t) {
         const int32_t eid = v.h2_eid[s];
         const uint32_t mycnt = v.h2_cnt[s];
         const int32_t* mine = v.corpus + v.h2_pos[s] + v.LL;
+        const uint32_t lo = v.grp_off[eid], hi = lo + v.grp_n[eid];
         int rank = 0;
-        uint32_t steps = 0;
-        for (uint32_t o = v.head[eid]; o != kEmpty && rank < v.FC && steps <= v.S; o = v.h2_next[o], ++steps) {
-            if (o == (uint32_t)s) continue;
-            const uint32_t c = v.h2_cnt[o];
+        for (uint32_t k = lo; k < hi && rank < v.FC; ++k) {
+            const uint32_t c = v.seg_cnt[k];
+            if (c < mycnt) continue;
             bool beats = c > mycnt;
-            if (c == mycnt) {
+            if (!beats) {
+                const uint32_t o = v.seg[k];
+                if (o == (uint32_t)s) continue;
                 const int32_t* other = v.corpus + v.h2_pos[o] + v.LL;
                 for (int j = 0; j < v.FL; ++j)
                     if (other[j] != mine[j]) { beats = other[j] < mine[j]; break; }
@@ -244,7 +276,7 @@ size_t fb_align(size_t x) { return (x + 255) / 256 * 256; }
 
 struct BuildLayout {
     uint32_t S;
-    size_t off_h1_pos, off_h1_cnt, off_h1_eid, off_uniq, off_h2_pos, off_h2_cnt, off_h2_eid, off_h2_next, off_head, total;
+    size_t off_h1_pos, off_h1_cnt, off_h1_eid, off_uniq, off_h2_pos, off_h2_cnt, off_h2_eid, off_seg, off_seg_cnt, off_grp, total;
 };
 
 cb_status fb_layout(const cb_frozen_config* c, int64_t n_tokens, BuildLayout* B) {
@@ -261,8 +293,9 @@ cb_status fb_layout(const cb_frozen_config* c, int64_t n_tokens, BuildLayout* B)
     B->off_h2_pos = o;  o = fb_align(o + S * 4);
     B->off_h2_cnt = o;  o = fb_align(o + S * 4);
     B->off_h2_eid = o;  o = fb_align(o + S * 4);
-    B->off_h2_next = o; o = fb_align(o + S * 4);
-    B->off_head = o;    o = fb_align(o + (size_t)c->LC * 4);
+    B->off_seg = o;     o = fb_align(o + S * 4);
+    B->off_seg_cnt = o; o = fb_align(o + S * 4);
+    B->off_grp = o;     o = fb_align(o + (size_t)c->LC * 4 * 3);
     B->total = o;
     return CB_OK;
 }
@@ -300,8 +333,8 @@ extern "C" cb_status cb_frozen_build(const cb_frozen_config* cfg, const int32_t*
     v.h1_pos = (uint32_t*)(base + B.off_h1_pos); v.h1_cnt = (uint32_t*)(base + B.off_h1_cnt); v.h1_eid = (int32_t*)(base + B.off_h1_eid);
     v.uniq = (uint32_t*)(base + B.off_uniq);
     v.h2_pos = (uint32_t*)(base + B.off_h2_pos); v.h2_cnt = (uint32_t*)(base + B.off_h2_cnt); v.h2_eid = (int32_t*)(base + B.off_h2_eid);
-    v.h2_next = (uint32_t*)(base + B.off_h2_next);
-    v.head = (uint32_t*)(base + B.off_head);
+    v.seg = (uint32_t*)(base + B.off_seg); v.seg_cnt = (uint32_t*)(base + B.off_seg_cnt);
+    v.grp_n = (uint32_t*)(base + B.off_grp); v.grp_off = v.grp_n + cfg->LC; v.grp_fill = v.grp_off + cfg->LC;
     v.S = B.S;
     v.corpus = dev_corpus;
     const int64_t M = n_tokens - cfg->LL - cfg->FL + 1;
@@ -322,8 +355,10 @@ extern "C" cb_status cb_frozen_build(const cb_frozen_config* cfg, const int32_t*
             }
         fb_place_leaders_kernel<<<grid, block, 0, st>>>(v, t);
         fb_count_followers_kernel<<<grid, block, 0, st>>>(v);
+        fb_group_scan_kernel<<<1, 1024, 0, st>>>(v);
+        fb_group_scatter_kernel<<<grid, block, 0, st>>>(v);
         fb_rank_followers_kernel<<<grid, block, 0, st>>>(v, t);
-        cb_count_launch(5 + 8 * (1 + cfg->LL));
+        cb_count_launch(7 + 8 * (1 + cfg->LL));
     }
     cb_count_launch(1);
     CB_CUDA(cudaGetLastError());

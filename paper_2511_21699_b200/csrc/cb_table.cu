@@ -95,26 +95,31 @@ __device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int
     if (pr.eid >= 0) {
         uint32_t* e = s.entries + (size_t)pr.eid * t.E;
         if (lane == 0) s.lstamp[pr.eid] = c;
-        const bool mine = lane < t.FC;
-        const uint32_t fs = mine ? e[t.LL + lane] : 0u;
-        bool match = mine && fs != 0u;
-        for (int j = 0; j < t.FL; ++j) {
-            const int32_t fj = __shfl_sync(CB_FULL, myfol, j);
-            if (mine && fs != 0u) match = match && ((int32_t)e[t.LL + t.FC + lane * t.FL + j] == fj);
-        }
-        const uint32_t mm = __ballot_sync(CB_FULL, match);
-        if (mm) {
-            if (t.refresh && lane == __ffs(mm) - 1) e[t.LL + lane] = c;
-        } else {
-            const uint32_t freem = __ballot_sync(CB_FULL, mine && fs == 0u);
-            int tgt;
-            if (freem) {
-                tgt = __ffs(freem) - 1;
-            } else {
-                const uint32_t g = __reduce_min_sync(CB_FULL, mine ? fs : 0xFFFFFFFFu);
-                tgt = __ffs(__ballot_sync(CB_FULL, mine && fs == g)) - 1;
-                cnt.fevict++;
+        // Lane l looks after followers l, l + 32, ...: one pass finds a stored copy of the follower, the lowest free place
+        // and the least recently inserted follower.
+        int match_f = -1, free_f = -1, lru_f = -1;
+        uint32_t lru_stamp = 0xFFFFFFFFu;
+        for (int base = 0; base < t.FC && match_f < 0; base += 32) {
+            const int f = base + lane;
+            const bool mine = f < t.FC;
+            const uint32_t fs = mine ? e[t.LL + f] : 0u;
+            bool match = mine && fs != 0u;
+            for (int j = 0; j < t.FL; ++j) {
+                const int32_t fj = __shfl_sync(CB_FULL, myfol, j);
+                if (match) match = ((int32_t)e[t.LL + t.FC + f * t.FL + j] == fj);
             }
+            const uint32_t mm = __ballot_sync(CB_FULL, match);
+            if (mm) { match_f = base + __ffs(mm) - 1; break; }
+            const uint32_t freem = __ballot_sync(CB_FULL, mine && fs == 0u);
+            if (free_f < 0 && freem) free_f = base + __ffs(freem) - 1;
+            const uint32_t g = __reduce_min_sync(CB_FULL, (mine && fs != 0u) ? fs : 0xFFFFFFFFu);
+            if (g < lru_stamp) { lru_stamp = g; lru_f = base + __ffs(__ballot_sync(CB_FULL, mine && fs == g)) - 1; }
+        }
+        if (match_f >= 0) {
+            if (t.refresh && lane == 0) e[t.LL + match_f] = c;
+        } else {
+            int tgt = free_f;
+            if (tgt < 0) { tgt = lru_f; cnt.fevict++; }
             if (lane < t.FL) e[t.LL + t.FC + tgt * t.FL + lane] = (uint32_t)myfol;
             if (lane == 0) e[t.LL + tgt] = c;
         }
@@ -132,7 +137,7 @@ __device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int
         } else {
             uint32_t* e = s.entries + (size_t)eid * t.E;
             if (lane < t.LL) e[lane] = (uint32_t)mykey;
-            if (lane < t.FC) e[t.LL + lane] = lane == 0 ? c : 0u;
+            for (int f = lane; f < t.FC; f += 32) e[t.LL + f] = f == 0 ? c : 0u;
             if (lane < t.FL) e[t.LL + t.FC + lane] = (uint32_t)myfol;
             if (lane == 0) {
                 s.lstamp[eid] = c;
@@ -191,7 +196,7 @@ struct DraftSmem {
     int32_t* fol;
 };
 
-__global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, int T, int crt, int max_depth, int NL, int FCmax,
+__global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, int T, int crt, int max_depth, int NL, int KF,
                                                        const int32_t* __restrict__ tokens, int64_t row_stride,
                                                        const int32_t* __restrict__ seq_len,
                                                        int32_t* __restrict__ o_tok, int32_t* __restrict__ o_par,
@@ -212,7 +217,7 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
     const int32_t* row = tokens + (size_t)b * row_stride;
     const int L = seq_len[b];
     const int W = (T + 31) >> 5;
-    const int FLFC = t.FL * FCmax;
+    const int FLFC = t.FL * KF;                               // staged followers per leaf: the KF best
     const uint32_t clock0 = s.hdr[0];
     const bool has_frozen = tf.index != nullptr;
 
@@ -267,18 +272,34 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
                     if (pr.eid >= 0) {
                         eid = pr.eid;
                         const uint32_t* e = ss.entries + (size_t)eid * tt.E;
-                        const uint32_t fs = lane < tt.FC ? e[tt.LL + lane] : 0u;
-                        // rank = number of followers with a larger stamp than mine (stamps are unique): more recently
-                        // inserted in the dynamic table, more frequent in the frozen one
-                        int rank = 0;
-                        for (int f = 0; f < tt.FC; ++f) {
-                            const uint32_t o = __shfl_sync(CB_FULL, fs, f);
-                            rank += (o > fs) ? 1 : 0;
+                        // Lane l holds the stamps of followers l, l + 32, ...  rank = number of followers with a larger stamp
+                        // than mine (stamps are unique): more recently inserted in the dynamic table, more frequent in the
+                        // frozen one.  Only the first KF ranks can ever be attached, so only they are staged.
+                        uint32_t fs[CB_MAX_FC / 32];
+#pragma unroll
+                        for (int c = 0; c < CB_MAX_FC / 32; ++c) fs[c] = (c * 32 + lane) < tt.FC ? e[tt.LL + c * 32 + lane] : 0u;
+                        int rank[CB_MAX_FC / 32];
+#pragma unroll
+                        for (int c = 0; c < CB_MAX_FC / 32; ++c) rank[c] = 0;
+#pragma unroll
+                        for (int c2 = 0; c2 < CB_MAX_FC / 32; ++c2) {
+                            if (c2 * 32 >= tt.FC) break;
+                            nf += __popc(__ballot_sync(CB_FULL, fs[c2] != 0u));
+                            const int lim = min(32, tt.FC - c2 * 32);
+                            for (int l = 0; l < lim; ++l) {
+                                const uint32_t o = __shfl_sync(CB_FULL, fs[c2], l);
+#pragma unroll
+                                for (int c = 0; c < CB_MAX_FC / 32; ++c) rank[c] += (o > fs[c]) ? 1 : 0;
+                            }
                         }
-                        nf = __popc(__ballot_sync(CB_FULL, fs != 0u));
-                        if (lane < tt.FC && fs != 0u)
-                            for (int j = 0; j < tt.FL; ++j)
-                                S.fol[li * FLFC + rank * tt.FL + j] = (int32_t)e[tt.LL + tt.FC + lane * tt.FL + j];
+                        nf = min(nf, KF);
+#pragma unroll
+                        for (int c = 0; c < CB_MAX_FC / 32; ++c) {
+                            const int f = c * 32 + lane;
+                            if (f < tt.FC && fs[c] != 0u && rank[c] < KF)
+                                for (int j = 0; j < tt.FL; ++j)
+                                    S.fol[li * FLFC + rank[c] * tt.FL + j] = (int32_t)e[tt.LL + tt.FC + f * tt.FL + j];
+                        }
                     }
                 }
                 if (lane == 0) { S.r_eid[li] = eid; S.r_nf[li] = nf; S.r_ok[li] = ok ? 1 : 0; S.r_stamp[li] = 0u; }
@@ -367,13 +388,23 @@ extern "C" cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t r
     const cb_config& c = ctx->cfg;
     const int T = c.max_nodes;
     const int NL = min(T, (T - 1) / c.FL + 1);
+    // A leaf can receive at most T - 1 followers (each adds a node), so no more than that many are staged per lookup.
     const int FCmax = ctx->has_frozen ? max(c.FC, ctx->frozen.FC) : c.FC;
-    const size_t smem = sizeof(int32_t) * ((size_t)3 * T + (size_t)7 * NL + (size_t)NL * c.FL * FCmax);
-    if (smem > 48 * 1024) return CB_ERR_UNSUPPORTED;
+    const int KF = max(1, min(FCmax, T - 1));
+    const size_t smem = sizeof(int32_t) * ((size_t)3 * T + (size_t)7 * NL + (size_t)NL * c.FL * KF);
+    if (smem > 200 * 1024) return CB_ERR_UNSUPPORTED;
+    if (smem > 48 * 1024) {
+        static size_t opted[64] = {0};                         // largest size opted into so far, per device
+        const int d = ctx->device & 63;
+        if (opted[d] < smem) {
+            CB_CUDA(cudaFuncSetAttribute(cb_draft_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            opted[d] = smem;
+        }
+    }
     const int threads = 32 * max(1, min(8, NL));
     CbTables tf = {};
     if (ctx->has_frozen) tf = ctx->frozen;
-    CB_CUDA(cb_launch_pdl(cb_draft_kernel, dim3(c.batch), dim3(threads), smem, (cudaStream_t)stream, ctx->tables, tf, T, c.crt, c.max_depth, NL, FCmax,
+    CB_CUDA(cb_launch_pdl(cb_draft_kernel, dim3(c.batch), dim3(threads), smem, (cudaStream_t)stream, ctx->tables, tf, T, c.crt, c.max_depth, NL, KF,
                           tokens, row_stride, seq_len, tree_tokens, tree_parent, tree_depth, tree_mask, n_nodes, ctx->d_status, ctx->d_counters));
     cb_count_launch(1);
     return CB_OK;

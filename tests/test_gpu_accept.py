@@ -64,7 +64,7 @@ def _run(cfg, dtype, full, sample_b, oracle, stride_pad=0):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("name,full", [("c1_tiny", True), ("c1_tiny", False), ("c2_7b", True), ("c4_13b_turns", False)])
+@pytest.mark.parametrize("name,full", [("c1_tiny", True), ("c1_tiny", False), ("c2_7b", True), ("c4_13b_turns", False), ("p_tuned", True)])
 def test_accept_logits_small(oracle, name, full, dtype):
     cfg = W.get_config(name)
     sample = range(cfg.batch) if cfg.batch <= 4 else [0, 1, 2, 31, 63]

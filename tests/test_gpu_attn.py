@@ -85,7 +85,7 @@ def test_attn_ragged_contexts_gqa(oracle, flags):
     _run(SMALL_GQA, oracle, False, _all, flags=flags, ctx_override=[0, 1, 16, 256, 299])
 
 
-@pytest.mark.parametrize("name", ["c2_7b", "c3_8b_gqa", "c4_13b_turns"])
+@pytest.mark.parametrize("name", ["c2_7b", "c3_8b_gqa", "c4_13b_turns", "p_tuned"])
 @pytest.mark.parametrize("full", [True, False])
 def test_attn_full_size_sampled(oracle, name, full):
     _run(W.get_config(name), oracle, full, _sampled(3, 3, 6))

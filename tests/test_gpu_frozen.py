@@ -59,7 +59,8 @@ def test_dual_draft_hand_trace_on_gpu(oracle):
 
 @pytest.mark.parametrize("name,steps,prompt,fLC,fFC", [("c1_tiny", 30, 8, 512, 8), ("c2_7b", 24, 48, 4096, 6),
                                                        ("c3_8b_gqa", 8, 32, 4096, 16), ("c4_13b_turns", 8, 64, 2048, 2),
-                                                       ("c1_evict256", 20, 300, 1024, 4)])
+                                                       ("c1_evict256", 20, 300, 1024, 4), ("p_tuned", 12, 64, 8192, 128),
+                                                       ("p_fc40_evict", 12, 600, 2048, 70)])
 def test_dual_draft_closed_loop(oracle, name, steps, prompt, fLC, fFC):
     """Cold start: a short prompt in the dynamic table, so that the frozen pass supplies much of each tree."""
     from paper_2511_21699_b200 import Cacheback
@@ -155,7 +156,8 @@ def _build_and_compare(oracle, corpus, LL, FL, LC, FC):
                                                  (2, 2, 500, 3, 12, 30000),      # tiny vocabulary: many equal counts
                                                  (3, 1, 777, 5, 6, 9000),
                                                  (4, 8, 2048, 2, 40, 15000),     # longest leader and follower
-                                                 (2, 3, 16, 1, 1000, 5000)])     # nearly every count is 1: ties decide
+                                                 (2, 3, 16, 1, 1000, 5000),      # nearly every count is 1: ties decide
+                                                 (1, 3, 4096, 128, 2000, 60000)])  # the paper's follower capacity
 def test_builder_matches_the_oracle(oracle, LL, FL, LC, FC, vocab, n):
     rng = np.random.default_rng(LL * 100 + FL)
     corpus = (rng.zipf(1.3, n) % vocab).astype(np.int32)

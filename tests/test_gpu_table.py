@@ -52,7 +52,8 @@ def _stream_targets(s, pos, n, tok, par, T, b, step):
 
 @pytest.mark.parametrize("name,steps", [("c1_tiny", 24), ("c2_7b", 24), ("c3_8b_gqa", 10), ("c4_13b_turns", 10),
                                         ("c5_70b_long", 4), ("c1_evict256", 24), ("c1_evict1024", 12),
-                                        ("c3_evict256", 10), ("c3_evict1024", 10)])
+                                        ("c3_evict256", 10), ("c3_evict1024", 10), ("p_tuned", 16),
+                                        ("p_fc40_evict", 16)])
 def test_update_draft_accept_closed_loop(oracle, name, steps):
     cfg = W.get_config(name)
     prob = Problem(cfg)
@@ -107,6 +108,8 @@ def test_update_draft_accept_closed_loop(oracle, name, steps):
     assert cnt["inserts"] > 0 and cnt["queries"] > 0
     if "evict" in name:
         assert cnt["leader_evictions"] > 0
+    if name.startswith("p_"):
+        assert cnt["follower_evictions"] > 0     # hot unigram leaders overflow even 128 followers
     if name in ("c1_tiny", "c3_8b_gqa", "c4_13b_turns", "c5_70b_long"):
         assert total_accept > 0                  # the drafter does get tokens accepted on these streams
 
