@@ -275,3 +275,34 @@ def kv_commit(k_pool, v_pool, block_table, ctx_len, k_tree, v_tree, n_accept, ac
             v_pool[page, pos % P] = v_tree[b, node]
         out[b] = ctx + m + 1
     return out
+
+
+def tree_add_branches(tok, par, dep, mask, n, max_depth, branches, branch_len):
+    """Drafts of another speculative-decoding method inserted as additional branches of the tree (paper, Conclusion: the
+    tree organisation lets other methods' predicted drafts be added as extra branches).
+
+    readings: a draft is a run of tokens that continues the sequence after the pending token, so it hangs below the root as
+    a chain; drafts are taken in the given order; a chain is cut where the tree's size cap T = len(tok) or the depth cap
+    would be exceeded (as table followers are) and a negative token ends it; branches are not compared with the nodes
+    already present.  A tree without a root (n = 0) takes nothing.
+    tok, par, dep: int32 [T]; mask: uint32 [T, W]; branches: int32 [K, Lmax]; branch_len: int32 [K].
+    Returns new copies (n, tok, par, dep, mask)."""
+    tok, par, dep = (np.array(x, dtype=np.int32, copy=True) for x in (tok, par, dep))
+    mask = np.array(mask, dtype=np.uint32, copy=True)
+    T = tok.shape[0]
+    n = int(n)
+    if n < 1:
+        return n, tok, par, dep, mask
+    branches = np.asarray(branches, dtype=np.int32)
+    for k in range(branches.shape[0]):
+        p = 0
+        for j in range(min(int(branch_len[k]), branches.shape[1])):
+            t = int(branches[k, j])
+            if t < 0 or n >= T or dep[p] >= max_depth:
+                break
+            tok[n], par[n], dep[n] = t, p, dep[p] + 1
+            mask[n] = mask[p]
+            mask[n, n // 32] |= np.uint32(1 << (n % 32))
+            p = n
+            n += 1
+    return n, tok, par, dep, mask
