@@ -131,6 +131,22 @@ cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, 
                         uint32_t* tree_mask, int32_t* n_nodes, void* stream);
 
 /*
+ * Extra branches from another drafter (Conclusion: because the drafts form a tree, the predicted drafts of other
+ * speculative-decoding methods can be inserted as additional branches).  Call it between cb_draft_tree and the
+ * verification pass.
+ *   branches    int32 [batch, n_branches, max_len]   each row a run of tokens continuing the sequence after its last token
+ *   branch_len  int32 [batch, n_branches]            tokens valid in each row (<= 0: none)
+ *   n_branches <= 64
+ * The tree arrays are those cb_draft_tree wrote and are extended in place.  For every sequence with a root, the branches
+ * are taken in order; each becomes a chain of new nodes below the root (node 0), cut where the tree would exceed max_nodes
+ * or a node max_depth, and ended by a negative token.  Branches are not compared with nodes already present.  The mask
+ * rows of the new nodes and n_nodes are updated.  The tables are not touched.
+ */
+cb_status cb_tree_add_branches(cb_ctx* ctx, const int32_t* branches, const int32_t* branch_len, int32_t n_branches,
+                               int32_t max_len, int32_t* tree_tokens, int32_t* tree_parent, int32_t* tree_depth,
+                               uint32_t* tree_mask, int32_t* n_nodes, void* stream);
+
+/*
  * Tree-masked attention over the paged KV cache (Section 3.2, "tree attention": a token attends only
  * to its ancestors in the draft tree; the cached context is fully visible).
  * With T = max_nodes, Hq / Hkv = n_q_heads / n_kv_heads, D = head_dim, P = page_size:

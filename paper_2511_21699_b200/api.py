@@ -181,6 +181,15 @@ class Cacheback:
                                       _ptr(tree["n_nodes"], torch.int32), _stream(stream)), "cb_draft_tree")
         return tree
 
+    def cb_tree_add_branches(self, tree, branches, branch_len, stream=None):
+        """branches int32 [batch, K, Lmax], branch_len int32 [batch, K]: extends `tree` in place."""
+        K, Lmax = int(branches.shape[1]), int(branches.shape[2])
+        _check(self.lib.cb_tree_add_branches(self._h, _ptr(branches, torch.int32), _ptr(branch_len, torch.int32), K, Lmax,
+                                             _ptr(tree["tokens"], torch.int32), _ptr(tree["parent"], torch.int32),
+                                             _ptr(tree["depth"], torch.int32), _ptr(tree["mask"], torch.int32),
+                                             _ptr(tree["n_nodes"], torch.int32), _stream(stream)), "cb_tree_add_branches")
+        return tree
+
     def cb_tree_attn(self, q, k_pool, v_pool, block_table, ctx_len, k_tree, v_tree, tree_mask, n_nodes, out=None,
                      lse=None, max_ctx=0, scale=0.0, stream=None):
         if out is None:

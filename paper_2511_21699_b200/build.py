@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 SO = os.path.join(HERE, "libcacheback.so")
-SOURCES = ["cb_api.cu", "cb_table.cu", "cb_accept.cu", "cb_kv.cu", "cb_frozen.cu", "cb_frozen_build.cu", "cb_attn.cu", "cb_attn_tc.cu"]
+SOURCES = ["cb_api.cu", "cb_table.cu", "cb_accept.cu", "cb_kv.cu", "cb_branches.cu", "cb_frozen.cu", "cb_frozen_build.cu", "cb_attn.cu", "cb_attn_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
