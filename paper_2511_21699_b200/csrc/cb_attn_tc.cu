@@ -252,19 +252,11 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
     const int RT = p.NPT * p.G;                               // rows of a row tile that exist
-    // The merge pass (like the next kernel of a step) is launched as a programmatic dependent: its blocks may take the SMs
-    // that this grid's CTAs leave and do their set-up there; they wait for this whole grid before they read any partial.
-    CB_PDL_ENTRY();
-
-    if (warp == 0) {
-        // this CTA's range of the global tile sequence
-        const long long tot = cb_sched_total(p, lane);
-        const long long g0 = cb_range_start(tot, p.nc, cta), g1 = cb_range_start(tot, p.nc, cta + 1);
-        int b0 = 0;
-        long long pre0 = 0;
-        if (g0 < g1) cb_sched_locate(p, g0, lane, &b0, &pre0);
-        if (lane == 0) { s_sched->g0 = g0; s_sched->g1 = g1; s_sched->b0 = b0; s_sched->pre0 = pre0; }
-    } else if (warp == 1) {
+    // Set-up that reads no input (TMEM allocation, barrier initialisation, descriptor prefetch) runs before the wait for the
+    // kernels earlier in the stream, so it overlaps their tail.  The merge pass (like the next kernel of a step) is launched as
+    // a programmatic dependent in turn: its blocks may take the SMs that this grid's CTAs leave and do their set-up there;
+    // they wait for this whole grid before they read any partial.
+    if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     } else if (warp == 2) {
@@ -279,6 +271,17 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             tma_prefetch_desc(&maps.k_pool); tma_prefetch_desc(&maps.v_pool); tma_prefetch_desc(&maps.q);
             tma_prefetch_desc(&maps.k_tree); tma_prefetch_desc(&maps.v_tree);
         }
+    }
+    CB_PDL_ENTRY();
+
+    if (warp == 0) {
+        // this CTA's range of the global tile sequence
+        const long long tot = cb_sched_total(p, lane);
+        const long long g0 = cb_range_start(tot, p.nc, cta), g1 = cb_range_start(tot, p.nc, cta + 1);
+        int b0 = 0;
+        long long pre0 = 0;
+        if (g0 < g1) cb_sched_locate(p, g0, lane, &b0, &pre0);
+        if (lane == 0) { s_sched->g0 = g0; s_sched->g1 = g1; s_sched->b0 = b0; s_sched->pre0 = pre0; }
     }
     tc_fence_before();
     __syncthreads();

@@ -243,97 +243,112 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
             __syncthreads();
         }
         while (true) {
-            const int nfront = sh_nfront, n_now = sh_n;
-            if (nfront == 0 || n_now >= T) break;
-            // (1) parallel lookups, one warp per leaf
-            for (int li = warp; li < nfront; li += nwarps) {
-                const int leaf = S.front[li];
-                const int d = S.dep[leaf];
-                // key = last LL tokens of (row[0 .. L-1) ++ root->leaf path); lane j < LL holds key[j]
-                int32_t mykey = 0;
-                bool ok = d < max_depth;
-                if (lane < t.LL) {
-                    const int back = t.LL - 1 - lane;         // distance from the leaf along the sequence
-                    if (back <= d) {
-                        int c = leaf;
-                        for (int k = 0; k < back; ++k) c = S.par[c];
-                        mykey = S.tok[c];
-                    } else {
-                        const int pos = L - 1 - (back - d);
-                        mykey = pos >= 0 ? row[pos] : -1;
+            const int nfront = sh_nfront;
+            if (nfront == 0 || sh_n >= T) break;
+            for (int li = tid; li < nfront; li += blockDim.x) S.r_stamp[li] = 0u;
+            if (tid == 0) sh_nnext = 0;
+            __syncthreads();
+            // With long follower lists the frontier is worked off in batches of one leaf per warp, lookups then replay, so that a
+            // level ends as soon as the tree is full (the first leaves of a level then usually take all the room).
+            const int BS = tt.FC > 32 ? nwarps : nfront;          // short follower lists: the whole frontier at once
+            for (int base = 0; base < nfront; base += BS) {
+                const int n_now = sh_n;
+                if (n_now >= T) break;
+                // (1) parallel lookups, one warp per leaf
+                for (int li = base + warp; li < min(nfront, base + BS); li += nwarps) {
+                    const int leaf = S.front[li];
+                    const int d = S.dep[leaf];
+                    // key = last LL tokens of (row[0 .. L-1) ++ root->leaf path); lane j < LL holds key[j]
+                    int32_t mykey = 0;
+                    bool ok = d < max_depth;
+                    if (lane < t.LL) {
+                        const int back = t.LL - 1 - lane;     // distance from the leaf along the sequence
+                        if (back <= d) {
+                            int c = leaf;
+                            for (int k = 0; k < back; ++k) c = S.par[c];
+                            mykey = S.tok[c];
+                        } else {
+                            const int pos = L - 1 - (back - d);
+                            mykey = pos >= 0 ? row[pos] : -1;
+                        }
                     }
-                }
-                ok = ok && __all_sync(CB_FULL, mykey >= 0);
-                int eid = -1, nf = 0;
-                if (ok) {
-                    const uint64_t h = warp_hash(tt, mykey);
-                    const Probe pr = tbl_find(tt, ss, mykey, h, lane);
-                    if (pr.eid == -2 && lane == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_PROBE_LIMIT);
-                    if (pr.eid >= 0) {
-                        eid = pr.eid;
-                        const uint32_t* e = ss.entries + (size_t)eid * tt.E;
-                        // Lane l holds the stamps of followers l, l + 32, ...  rank = number of followers with a larger stamp
-                        // than mine (stamps are unique): more recently inserted in the dynamic table, more frequent in the
-                        // frozen one.  Only the first KF ranks can ever be attached, so only they are staged.
-                        uint32_t fs[CB_MAX_FC / 32];
+                    ok = ok && __all_sync(CB_FULL, mykey >= 0);
+                    int eid = -1, nf = 0;
+                    if (ok) {
+                        const uint64_t h = warp_hash(tt, mykey);
+                        const Probe pr = tbl_find(tt, ss, mykey, h, lane);
+                        if (pr.eid == -2 && lane == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_PROBE_LIMIT);
+                        if (pr.eid >= 0) {
+                            eid = pr.eid;
+                            const uint32_t* e = ss.entries + (size_t)eid * tt.E;
+                            // Lane l holds the stamps of followers l, l + 32, ...  The followers are wanted by falling stamp
+                            // (most recently inserted first in the dynamic table, most frequent first in the frozen one),
+                            // and only as many as the tree still has room for: they are picked one by one with a warp-wide
+                            // maximum (stamps are unique) and staged in that order.
+                            uint32_t fs[CB_MAX_FC / 32];
 #pragma unroll
-                        for (int c = 0; c < CB_MAX_FC / 32; ++c) fs[c] = (c * 32 + lane) < tt.FC ? e[tt.LL + c * 32 + lane] : 0u;
-                        int rank[CB_MAX_FC / 32];
+                            for (int c = 0; c < CB_MAX_FC / 32; ++c) {
+                                fs[c] = (c * 32 + lane) < tt.FC ? e[tt.LL + c * 32 + lane] : 0u;
+                                nf += __popc(__ballot_sync(CB_FULL, fs[c] != 0u));
+                            }
+                            nf = min(nf, min(KF, (leaf == 0 ? max(1, T - crt) : T) - n_now));
+                            int rank[CB_MAX_FC / 32];
 #pragma unroll
-                        for (int c = 0; c < CB_MAX_FC / 32; ++c) rank[c] = 0;
+                            for (int c = 0; c < CB_MAX_FC / 32; ++c) rank[c] = -1;
+                            for (int r = 0; r < nf; ++r) {
+                                uint32_t m = fs[0];
 #pragma unroll
-                        for (int c2 = 0; c2 < CB_MAX_FC / 32; ++c2) {
-                            if (c2 * 32 >= tt.FC) break;
-                            nf += __popc(__ballot_sync(CB_FULL, fs[c2] != 0u));
-                            const int lim = min(32, tt.FC - c2 * 32);
-                            for (int l = 0; l < lim; ++l) {
-                                const uint32_t o = __shfl_sync(CB_FULL, fs[c2], l);
+                                for (int c = 1; c < CB_MAX_FC / 32; ++c) m = max(m, fs[c]);
+                                const uint32_t g = __reduce_max_sync(CB_FULL, m);
 #pragma unroll
-                                for (int c = 0; c < CB_MAX_FC / 32; ++c) rank[c] += (o > fs[c]) ? 1 : 0;
+                                for (int c = 0; c < CB_MAX_FC / 32; ++c)
+                                    if (fs[c] == g) { rank[c] = r; fs[c] = 0u; }
+                            }
+                            // every lane copies the tokens of its picked followers
+#pragma unroll
+                            for (int c = 0; c < CB_MAX_FC / 32; ++c) {
+                                if (rank[c] >= 0) {
+                                    const int f = c * 32 + lane;
+                                    for (int j = 0; j < tt.FL; ++j)
+                                        S.fol[li * FLFC + rank[c] * tt.FL + j] = (int32_t)e[tt.LL + tt.FC + f * tt.FL + j];
+                                }
                             }
                         }
-                        nf = min(nf, KF);
-#pragma unroll
-                        for (int c = 0; c < CB_MAX_FC / 32; ++c) {
-                            const int f = c * 32 + lane;
-                            if (f < tt.FC && fs[c] != 0u && rank[c] < KF)
-                                for (int j = 0; j < tt.FL; ++j)
-                                    S.fol[li * FLFC + rank[c] * tt.FL + j] = (int32_t)e[tt.LL + tt.FC + f * tt.FL + j];
+                    }
+                    if (lane == 0) { S.r_eid[li] = eid; S.r_nf[li] = nf; S.r_ok[li] = ok ? 1 : 0; }
+                }
+                __syncthreads();
+                // (2) sequential replay of the breadth-first order.  A query at the root (the only leaf of level 1) is issued,
+                // and its followers attached, while the tree has fewer than max(1, T - crt) nodes; any other while fewer than T.
+                if (tid == 0) {
+                    int n = n_now, q = 0, hits = 0, nn = sh_nnext;
+                    const int lend = min(nfront, base + BS);
+                    for (int l2 = base; l2 < lend; ++l2) {
+                        if (n >= T) break;
+                        const int leaf = S.front[l2];
+                        const int cap = leaf == 0 ? max(1, T - crt) : T;
+                        if (n >= cap) continue;
+                        if (!S.r_ok[l2]) continue;
+                        ++q;                                    // this query is issued: the dynamic table's clock ticks
+                        if (S.r_eid[l2] < 0) continue;
+                        ++hits;
+                        if (pass == 0) S.r_stamp[l2] = clock0 + (uint32_t)(sh_q + q);
+                        for (int f = 0; f < S.r_nf[l2]; ++f) {
+                            if (n >= cap) break;
+                            int p = leaf, k = 0;
+                            for (int j = 0; j < t.FL; ++j) {
+                                if (n >= cap || S.dep[p] >= max_depth) break;
+                                S.tok[n] = S.fol[l2 * FLFC + f * t.FL + j];
+                                S.par[n] = p; S.dep[n] = S.dep[p] + 1; p = n; ++n; ++k;
+                            }
+                            if (k == t.FL) S.next[nn++] = p;
                         }
                     }
+                    sh_n = n; sh_nnext = nn;
+                    if (pass == 0) { sh_q += q; sh_hits += hits; } else { sh_fq += q; sh_fhits += hits; }
                 }
-                if (lane == 0) { S.r_eid[li] = eid; S.r_nf[li] = nf; S.r_ok[li] = ok ? 1 : 0; S.r_stamp[li] = 0u; }
+                __syncthreads();
             }
-            __syncthreads();
-            // (2) sequential replay of the breadth-first order.  A query at the root (the only leaf of level 1) is issued,
-            // and its followers attached, while the tree has fewer than max(1, T - crt) nodes; any other while fewer than T.
-            if (tid == 0) {
-                int n = n_now, q = 0, hits = 0, nn = 0;
-                for (int li = 0; li < nfront; ++li) {
-                    if (n >= T) break;
-                    const int leaf = S.front[li];
-                    const int cap = leaf == 0 ? max(1, T - crt) : T;
-                    if (n >= cap) continue;
-                    if (!S.r_ok[li]) continue;
-                    ++q;                                        // this query is issued: the dynamic table's clock ticks
-                    if (S.r_eid[li] < 0) continue;
-                    ++hits;
-                    if (pass == 0) S.r_stamp[li] = clock0 + (uint32_t)(sh_q + q);
-                    for (int f = 0; f < S.r_nf[li]; ++f) {
-                        if (n >= cap) break;
-                        int p = leaf, k = 0;
-                        for (int j = 0; j < t.FL; ++j) {
-                            if (n >= cap || S.dep[p] >= max_depth) break;
-                            S.tok[n] = S.fol[li * FLFC + f * t.FL + j];
-                            S.par[n] = p; S.dep[n] = S.dep[p] + 1; p = n; ++n; ++k;
-                        }
-                        if (k == t.FL) S.next[nn++] = p;
-                    }
-                }
-                sh_n = n; sh_nnext = nn;
-                if (pass == 0) { sh_q += q; sh_hits += hits; } else { sh_fq += q; sh_fhits += hits; }
-            }
-            __syncthreads();
             // (3) stamp the leaders the sequential order reached; publish the next frontier
             if (pass == 0)
                 for (int li = tid; li < nfront; li += blockDim.x)
