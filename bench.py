@@ -43,8 +43,8 @@ def parse():
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one cb_attn_tc_kernel launch, from the ncu capture
 # summarised in profiles/cb_attn_tc_kernel_<workload>.md.  It is reported only while the kernel sources still hash to the
 # captured ones; after any change to them the figure is stale and `traffic` is null until the capture is redone.
-ATTN_TRAFFIC = {"sources_sha1": "3b0af9cc8abea278d1aafd0e767d0652980f9456",
-                "bytes_per_launch": {"c2_7b": 70.08e6, "c3_8b_gqa": 589.2e6, "c4_13b_turns": 2792.1e6}}
+ATTN_TRAFFIC = {"sources_sha1": "5d36805bcc9a40a99a44b6f5c42595303f7719d2",
+                "bytes_per_launch": {"c2_7b": 69.95e6, "c3_8b_gqa": 589.6e6, "c4_13b_turns": 2792.5e6}}
 
 
 def attn_sources_sha1():
