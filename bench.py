@@ -279,7 +279,7 @@ def run_ours(args, rank, world, local_rank):
     assert int((lens - prefill).min()) > ADVANCE * total + T, "stream too short for this many steps"
     n_old = dev(np.stack([prefill + ADVANCE * s for s in range(total)]).astype(np.int32))
     n_new = dev(np.stack([prefill + ADVANCE * (s + 1) for s in range(total)]).astype(np.int32))
-    cb.cb_update(toks_d, dev(np.zeros(B, np.int32)), dev(prefill))          # prompt initialisation, untimed
+    cb.cb_update_bulk(toks_d, dev(np.zeros(B, np.int32)), dev(prefill))     # prompt initialisation, untimed
     frozen_info = None
     if args.frozen > 0:
         # Stand-in for the paper's corpus sample: streams of the workload's own token distribution under other seeds.

@@ -111,6 +111,15 @@ cb_status cb_update(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, cons
                     const int32_t* n_new, void* stream);
 
 /*
+ * cb_update for long runs of new tokens (Section 3.3: the dynamic table is initialised with a sliding window over the
+ * prompt).  Same arguments, same resulting tables, clocks and counters as cb_update; the work of one sequence is spread
+ * over many warps where that cannot change the result (no leader can be evicted during the run: leaders stored + windows
+ * <= LC, and at least 64 windows), and done by one warp in order otherwise.  Two launches.
+ */
+cb_status cb_update_bulk(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* n_old,
+                         const int32_t* n_new, void* stream);
+
+/*
  * Draft-tree growth (Section 3.2).
  *   tokens, row_stride  as in cb_update;  seq_len int32 [batch] = tokens valid per sequence
  * Node 0 is the last token of the sequence (the one token whose K/V is not cached yet).  Level 1

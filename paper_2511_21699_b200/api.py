@@ -167,6 +167,10 @@ class Cacheback:
         _check(self.lib.cb_update(self._h, _ptr(tokens, torch.int32), tokens.stride(0), _ptr(n_old, torch.int32),
                                   _ptr(n_new, torch.int32), _stream(stream)), "cb_update")
 
+    def cb_update_bulk(self, tokens, n_old, n_new, stream=None):
+        _check(self.lib.cb_update_bulk(self._h, _ptr(tokens, torch.int32), tokens.stride(0), _ptr(n_old, torch.int32),
+                                       _ptr(n_new, torch.int32), _stream(stream)), "cb_update_bulk")
+
     def alloc_tree(self):
         B, T = self.cfg.batch, self.cfg.max_nodes
         i32 = dict(dtype=torch.int32, device=self.device)

@@ -41,6 +41,7 @@ cb_status cb_compute_layout(const cb_config* c, CbLayout* L) {
     L->off_counters = o; o = align_up(o + CB_NUM_COUNTERS * 8, 256);
     L->off_rowmax = o;   o = align_up(o + B * (size_t)c->max_nodes * 8, 256);
     L->off_ticket = o;   o = align_up(o + B * 4, 256);
+    L->off_bulk_plan = o; o = align_up(o + B * 16, 256);
     L->attn_max_units = CB_ATTN_MAX_UNITS;
     L->attn_part_floats = (size_t)L->attn_max_units * 128 * ((size_t)c->head_dim + 4);
     L->off_attn_part = o; o = align_up(o + L->attn_part_floats * 4, 256);
@@ -86,6 +87,7 @@ extern "C" cb_status cb_create(const cb_config* cfg, void* dev_workspace, size_t
     c->d_counters = (unsigned long long*)(c->ws + L.off_counters);
     c->d_rowmax = (unsigned long long*)(c->ws + L.off_rowmax);
     c->d_ticket = (uint32_t*)(c->ws + L.off_ticket);
+    c->d_bulk_plan = (uint32_t*)(c->ws + L.off_bulk_plan);
     c->d_attn_part = (float*)(c->ws + L.off_attn_part);
     c->attn_part_floats = L.attn_part_floats;
     c->attn_max_units = L.attn_max_units;

@@ -75,6 +75,7 @@ struct cb_ctx {
     unsigned long long* d_counters;  // [CB_NUM_COUNTERS]
     unsigned long long* d_rowmax;    // [batch * max_nodes] packed (value, index) maxima, zero between calls
     uint32_t* d_ticket;     // [batch] CTAs-finished counters, zero between calls
+    uint32_t* d_bulk_plan;  // [batch][4] per-sequence plan of cb_update_bulk
     float* d_attn_part;     // partial outputs of units shared between CTAs
     size_t attn_part_floats;
     int attn_max_units;     // partial row tiles available
@@ -83,7 +84,7 @@ struct cb_ctx {
 
 struct CbLayout {
     uint32_t nslots, E;
-    size_t off_hdr, off_index, off_lstamp, off_entries, off_status, off_counters, off_rowmax, off_ticket,
+    size_t off_hdr, off_index, off_lstamp, off_entries, off_status, off_counters, off_rowmax, off_ticket, off_bulk_plan,
         off_attn_part, attn_part_floats, total;
     int attn_max_units;
 };

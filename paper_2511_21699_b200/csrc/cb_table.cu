@@ -23,14 +23,15 @@ __device__ __forceinline__ Probe tbl_find(const CbTables& t, const CbSeq& s, int
     uint32_t bucket = cb_hash_bucket(h, t.nslots);
     for (uint32_t p = 0; p < nb; ++p) {
         r.probes = p + 1;
-        const uint32_t w = s.index[bucket * 32 + lane];
+        // read through to L2: in the bulk update other SMs publish index words and entries while this warp probes
+        const uint32_t w = __ldcg(&s.index[bucket * 32 + lane]);
         uint32_t cand = __ballot_sync(CB_FULL, w != CB_IDX_EMPTY && w != CB_IDX_TOMB && (w >> CB_EID_BITS) == tag);
         while (cand) {
             const int l = __ffs(cand) - 1;
             cand &= cand - 1;
             const uint32_t eid = __shfl_sync(CB_FULL, w, l) & CB_EID_MASK;
             bool eq = true;
-            if (lane < t.LL) eq = ((int32_t)s.entries[(size_t)eid * t.E + lane] == mykey);
+            if (lane < t.LL) eq = ((int32_t)__ldcg(&s.entries[(size_t)eid * t.E + lane]) == mykey);
             if (__all_sync(CB_FULL, eq)) { r.eid = (int)eid; r.slot = bucket * 32 + l; return r; }
         }
         const uint32_t fr = __ballot_sync(CB_FULL, w == CB_IDX_EMPTY || w == CB_IDX_TOMB);
@@ -84,6 +85,39 @@ __device__ int tbl_evict_lru(const CbTables& t, const CbSeq& s, int lane, uint32
 
 struct TblCounters { uint32_t inserts, levict, fevict, maxprobe; };
 
+// Follower list of an existing leader (Section 3.1): a stored copy of the follower is refreshed, otherwise the follower takes
+// the lowest free place or replaces the least recently inserted one.  e = the leader's entry, c = this operation's stamp.
+__device__ __forceinline__ void tbl_put_follower(const CbTables& t, uint32_t* e, int32_t myfol, uint32_t c, int lane, TblCounters& cnt) {
+    // Lane l looks after followers l, l + 32, ...: one pass finds a stored copy of the follower, the lowest free place
+    // and the least recently inserted follower.
+    int match_f = -1, free_f = -1, lru_f = -1;
+    uint32_t lru_stamp = 0xFFFFFFFFu;
+    for (int base = 0; base < t.FC && match_f < 0; base += 32) {
+        const int f = base + lane;
+        const bool mine = f < t.FC;
+        const uint32_t fs = mine ? e[t.LL + f] : 0u;
+        bool match = mine && fs != 0u;
+        for (int j = 0; j < t.FL; ++j) {
+            const int32_t fj = __shfl_sync(CB_FULL, myfol, j);
+            if (match) match = ((int32_t)e[t.LL + t.FC + f * t.FL + j] == fj);
+        }
+        const uint32_t mm = __ballot_sync(CB_FULL, match);
+        if (mm) { match_f = base + __ffs(mm) - 1; break; }
+        const uint32_t freem = __ballot_sync(CB_FULL, mine && fs == 0u);
+        if (free_f < 0 && freem) free_f = base + __ffs(freem) - 1;
+        const uint32_t g = __reduce_min_sync(CB_FULL, (mine && fs != 0u) ? fs : 0xFFFFFFFFu);
+        if (g < lru_stamp) { lru_stamp = g; lru_f = base + __ffs(__ballot_sync(CB_FULL, mine && fs == g)) - 1; }
+    }
+    if (match_f >= 0) {
+        if (t.refresh && lane == 0) e[t.LL + match_f] = c;
+    } else {
+        int tgt = free_f;
+        if (tgt < 0) { tgt = lru_f; cnt.fevict++; }
+        if (lane < t.FL) e[t.LL + t.FC + tgt * t.FL + lane] = (uint32_t)myfol;
+        if (lane == 0) e[t.LL + tgt] = c;
+    }
+}
+
 // One insertion (Section 3.1). mykey = leader[lane] (lane < LL), myfol = follower[lane] (lane < FL).
 __device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int32_t myfol, uint32_t& clock,
                            uint32_t& count, int lane, uint32_t* status, TblCounters& cnt) {
@@ -95,34 +129,7 @@ __device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int
     if (pr.eid >= 0) {
         uint32_t* e = s.entries + (size_t)pr.eid * t.E;
         if (lane == 0) s.lstamp[pr.eid] = c;
-        // Lane l looks after followers l, l + 32, ...: one pass finds a stored copy of the follower, the lowest free place
-        // and the least recently inserted follower.
-        int match_f = -1, free_f = -1, lru_f = -1;
-        uint32_t lru_stamp = 0xFFFFFFFFu;
-        for (int base = 0; base < t.FC && match_f < 0; base += 32) {
-            const int f = base + lane;
-            const bool mine = f < t.FC;
-            const uint32_t fs = mine ? e[t.LL + f] : 0u;
-            bool match = mine && fs != 0u;
-            for (int j = 0; j < t.FL; ++j) {
-                const int32_t fj = __shfl_sync(CB_FULL, myfol, j);
-                if (match) match = ((int32_t)e[t.LL + t.FC + f * t.FL + j] == fj);
-            }
-            const uint32_t mm = __ballot_sync(CB_FULL, match);
-            if (mm) { match_f = base + __ffs(mm) - 1; break; }
-            const uint32_t freem = __ballot_sync(CB_FULL, mine && fs == 0u);
-            if (free_f < 0 && freem) free_f = base + __ffs(freem) - 1;
-            const uint32_t g = __reduce_min_sync(CB_FULL, (mine && fs != 0u) ? fs : 0xFFFFFFFFu);
-            if (g < lru_stamp) { lru_stamp = g; lru_f = base + __ffs(__ballot_sync(CB_FULL, mine && fs == g)) - 1; }
-        }
-        if (match_f >= 0) {
-            if (t.refresh && lane == 0) e[t.LL + match_f] = c;
-        } else {
-            int tgt = free_f;
-            if (tgt < 0) { tgt = lru_f; cnt.fevict++; }
-            if (lane < t.FL) e[t.LL + t.FC + tgt * t.FL + lane] = (uint32_t)myfol;
-            if (lane == 0) e[t.LL + tgt] = c;
-        }
+        tbl_put_follower(t, e, myfol, c, lane, cnt);
     } else if (pr.eid == -1) {
         int eid;
         if (count < (uint32_t)t.LC) {
@@ -172,6 +179,136 @@ __global__ void __launch_bounds__(128) cb_update_kernel(CbTables t, int B, const
     }
     if (lane == 0) {
         s.hdr[0] = clock; s.hdr[1] = count;
+        if (cnt.inserts) atomicAdd(&counters[CB_CNT_INSERTS], (unsigned long long)cnt.inserts);
+        if (cnt.levict) atomicAdd(&counters[CB_CNT_LEADER_EVICTIONS], (unsigned long long)cnt.levict);
+        if (cnt.fevict) atomicAdd(&counters[CB_CNT_FOLLOWER_EVICTIONS], (unsigned long long)cnt.fevict);
+        if (cnt.maxprobe) atomicMax(&counters[CB_CNT_MAX_PROBE], (unsigned long long)cnt.maxprobe);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Bulk update (prompt initialisation and other long runs of new tokens): many warps per sequence.
+//
+// The result of a run of insertions depends on their order only within one leader (its recency and its follower list)
+// and, across leaders, through leader eviction.  Stamps are a function of the window's position (the clock ticks once per
+// window), so when no leader can be evicted during the run (leaders stored + windows <= LC) the windows may be dealt out
+// to warps by a hash of their leader: every leader is handled by one warp, in increasing position, exactly as the
+// sequential kernel would, and different leaders touch disjoint entries.  What the warps share is the leader counter
+// (atomicAdd hands out entry ids) and the index, whose slots are claimed with atomicCAS; an entry is complete before its
+// index word is published.  A plan kernel takes that decision once per sequence, before any warp changes the table;
+// sequences that do not qualify (short runs, possible eviction) are done by their first warp alone, in order.
+struct BulkPlan { uint32_t parallel, clock0, first, nwin; };
+
+__global__ void cb_bulk_plan_kernel(CbTables t, int B, const int32_t* __restrict__ n_old, const int32_t* __restrict__ n_new,
+                                    BulkPlan* plan) {
+    CB_PDL_ENTRY();
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const CbSeq s = cb_seq(t, b);
+    const int w = t.LL + t.FL;
+    const int first = max(0, n_old[b] - w + 1);
+    const int nwin = max(0, n_new[b] - w + 1 - first);
+    BulkPlan p;
+    p.clock0 = s.hdr[0];
+    p.first = (uint32_t)first;
+    p.nwin = (uint32_t)nwin;
+    p.parallel = (nwin >= 64 && (unsigned long long)s.hdr[1] + (unsigned long long)nwin <= (unsigned long long)t.LC) ? 1u : 0u;
+    if (p.parallel) s.hdr[0] = p.clock0 + (uint32_t)nwin;      // the clock after the run; the warps take stamps from positions
+    plan[b] = p;
+}
+
+// One insertion of the parallel path: c is the operation's stamp; no leader is ever evicted here.
+__device__ void tbl_insert_shared(const CbTables& t, const CbSeq& s, int32_t mykey, int32_t myfol, uint32_t c, int lane,
+                                  uint32_t* status, TblCounters& cnt) {
+    cnt.inserts++;
+    const uint64_t h = warp_hash(t, mykey);
+    const uint32_t tagword = cb_hash_tag(h) << CB_EID_BITS;
+    int eid = -1;
+    for (int attempt = 0; attempt < 64; ++attempt) {            // a claim can lose its slot to another warp's leader: look again
+        const Probe pr = tbl_find(t, s, mykey, h, lane);
+        cnt.maxprobe = max(cnt.maxprobe, pr.probes);
+        if (pr.eid >= 0) {
+            uint32_t* e = s.entries + (size_t)pr.eid * t.E;
+            if (lane == 0) s.lstamp[pr.eid] = c;
+            tbl_put_follower(t, e, myfol, c, lane, cnt);
+            __syncwarp();
+            return;
+        }
+        if (pr.eid != -1 || pr.free_slot == 0xFFFFFFFFu) break;
+        if (eid < 0) {
+            // new leader: take an entry, fill it, then publish it
+            uint32_t got = 0;
+            if (lane == 0) got = atomicAdd(&s.hdr[1], 1u);
+            got = __shfl_sync(CB_FULL, got, 0);
+            if (got >= (uint32_t)t.LC) break;                  // excluded by the plan
+            eid = (int)got;
+            uint32_t* e = s.entries + (size_t)eid * t.E;
+            if (lane < t.LL) e[lane] = (uint32_t)mykey;
+            for (int f = lane; f < t.FC; f += 32) e[t.LL + f] = f == 0 ? c : 0u;
+            if (lane < t.FL) e[t.LL + t.FC + lane] = (uint32_t)myfol;
+            if (lane == 0) s.lstamp[eid] = c;
+            __threadfence();
+            __syncwarp();
+        }
+        uint32_t old = 0;
+        if (lane == 0) old = atomicCAS(&s.index[pr.free_slot], CB_IDX_EMPTY, tagword | (uint32_t)eid);
+        old = __shfl_sync(CB_FULL, old, 0);
+        if (old == CB_IDX_EMPTY) return;
+        if (old == CB_IDX_TOMB) {                              // a deleted slot is as good as an empty one
+            if (lane == 0) old = atomicCAS(&s.index[pr.free_slot], CB_IDX_TOMB, tagword | (uint32_t)eid);
+            old = __shfl_sync(CB_FULL, old, 0);
+            if (old == CB_IDX_TOMB) return;
+        }
+    }
+    if (lane == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_PROBE_LIMIT);
+}
+
+__global__ void __launch_bounds__(256) cb_update_bulk_kernel(CbTables t, int B, int WPS, const int32_t* __restrict__ tokens, int64_t row_stride,
+                                                             const int32_t* __restrict__ n_old, const int32_t* __restrict__ n_new,
+                                                             const BulkPlan* __restrict__ plan, uint32_t* status, unsigned long long* counters) {
+    CB_PDL_ENTRY();
+    const int lane = threadIdx.x & 31;
+    const int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int b = gw / WPS, wi = gw % WPS;
+    if (b >= B) return;
+    const CbSeq s = cb_seq(t, b);
+    const BulkPlan pl = plan[b];
+    const int32_t* row = tokens + (size_t)b * row_stride;
+    TblCounters cnt = {0, 0, 0, 0};
+    if (!pl.parallel) {
+        if (wi != 0) return;
+        uint32_t clock = s.hdr[0], count = s.hdr[1];
+        for (uint32_t k = 0; k < pl.nwin; ++k) {
+            const int i = (int)(pl.first + k);
+            const int32_t mykey = lane < t.LL ? row[i + lane] : 0;
+            const int32_t myfol = lane < t.FL ? row[i + t.LL + lane] : 0;
+            tbl_insert(t, s, mykey, myfol, clock, count, lane, status, cnt);
+        }
+        if (lane == 0) { s.hdr[0] = clock; s.hdr[1] = count; }
+    } else {
+        // 32 windows at a time: every lane hashes one leader, the warp keeps those that are its own and inserts them in order
+        for (uint32_t k0 = 0; k0 < pl.nwin; k0 += 32) {
+            const uint32_t k = k0 + lane;
+            bool mine = false;
+            if (k < pl.nwin) {
+                const int i = (int)(pl.first + k);
+                int32_t k4[4] = {0, 0, 0, 0};
+                for (int j = 0; j < t.LL; ++j) k4[j] = row[i + j];
+                const uint64_t h = cb_hash4(k4[0], k4[1], k4[2], k4[3], t.LL);
+                mine = (uint32_t)((h >> 17) % (uint64_t)WPS) == (uint32_t)wi;
+            }
+            uint32_t todo = __ballot_sync(CB_FULL, mine);
+            while (todo) {
+                const int l = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const int i = (int)(pl.first + k0 + l);
+                const int32_t mykey = lane < t.LL ? row[i + lane] : 0;
+                const int32_t myfol = lane < t.FL ? row[i + t.LL + lane] : 0;
+                tbl_insert_shared(t, s, mykey, myfol, pl.clock0 + k0 + (uint32_t)l + 1u, lane, status, cnt);
+            }
+        }
+    }
+    if (lane == 0) {
         if (cnt.inserts) atomicAdd(&counters[CB_CNT_INSERTS], (unsigned long long)cnt.inserts);
         if (cnt.levict) atomicAdd(&counters[CB_CNT_LEADER_EVICTIONS], (unsigned long long)cnt.levict);
         if (cnt.fevict) atomicAdd(&counters[CB_CNT_FOLLOWER_EVICTIONS], (unsigned long long)cnt.fevict);
@@ -392,6 +529,22 @@ extern "C" cb_status cb_update(cb_ctx* ctx, const int32_t* tokens, int64_t row_s
     CB_CUDA(cb_launch_pdl(cb_update_kernel, dim3((B + wpb - 1) / wpb), dim3(wpb * 32), 0, (cudaStream_t)stream, ctx->tables, B, tokens, row_stride,
                           n_old, n_new, ctx->d_status, ctx->d_counters));
     cb_count_launch(1);
+    return CB_OK;
+}
+
+extern "C" cb_status cb_update_bulk(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* n_old,
+                                    const int32_t* n_new, void* stream) {
+    CB_CHECK_ARG(ctx && tokens && n_old && n_new && row_stride >= 1);
+    const int B = ctx->cfg.batch;
+    // enough warps per sequence to fill the GPU at small batch, fewer at large batch
+    int wps = 1;
+    while (wps < 64 && (long long)B * wps * 2 <= (long long)ctx->num_sms * 16) wps *= 2;
+    BulkPlan* plan = reinterpret_cast<BulkPlan*>(ctx->d_bulk_plan);
+    CB_CUDA(cb_launch_pdl(cb_bulk_plan_kernel, dim3((B + 127) / 128), dim3(128), 0, (cudaStream_t)stream, ctx->tables, B, n_old, n_new, plan));
+    const long long warps = (long long)B * wps;
+    CB_CUDA(cb_launch_pdl(cb_update_bulk_kernel, dim3((unsigned)((warps + 7) / 8)), dim3(256), 0, (cudaStream_t)stream, ctx->tables, B, wps, tokens,
+                          row_stride, n_old, n_new, (const BulkPlan*)plan, ctx->d_status, ctx->d_counters));
+    cb_count_launch(2);
     return CB_OK;
 }
 
