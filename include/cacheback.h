@@ -270,7 +270,7 @@ cb_status cb_kv_commit(cb_ctx* ctx, const cb_kv_commit_args* args, void* stream)
  * than max_nodes; max_depth; a follower that does not fit is cut short).  Frozen followers are not compared with the
  * branches already present.  Frozen queries touch no recency and are counted in CB_CNT_FROZEN_QUERIES / _HITS.
  *
- * Offline construction (Section 4.1: from a corpus sample, the LC most frequent n-grams of length LL become the leaders,
+ * Offline construction (Section 4: from a corpus sample, the LC most frequent n-grams of length LL become the leaders,
  * and each leader keeps the FC most frequent n-grams of length FL that follow it).
  *   cb_frozen_build   counts on the GPU.  dev_corpus int32 [n_tokens] (device, ids >= 0, one token stream,
  *                     n_tokens <= 2^30); an occurrence is counted where LL + FL tokens are available, so every leader

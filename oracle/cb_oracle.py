@@ -140,7 +140,7 @@ class OracleTable:
 
 
 def frozen_build(corpus, LL, FL, LC, FC):
-    """Offline construction of the frozen table (paper Section 4.1, experimental set-up): the LC most frequent n-grams of
+    """Offline construction of the frozen table (paper Section 4, experimental set-up): the LC most frequent n-grams of
     length LL become the leaders; each leader keeps the FC most frequent n-grams of length FL that follow it.
 
     readings: the corpus is one token stream; an occurrence counts where LL + FL tokens are available, so every leader

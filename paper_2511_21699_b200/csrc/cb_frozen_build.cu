@@ -1,4 +1,4 @@
-// Offline construction of a frozen table from a token corpus on the GPU (Section 4.1: the most frequent LC n-grams of
+// Offline construction of a frozen table from a token corpus on the GPU (Section 4: the most frequent LC n-grams of
 // length LL become the leaders; each keeps the FC most frequent n-grams of length FL that follow it).
 //
 // A window is LL + FL consecutive tokens; the corpus of N tokens has M = N - LL - FL + 1 of them.  Everything is counting

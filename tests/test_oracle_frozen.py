@@ -1,4 +1,4 @@
-"""Pins for the oracle's frozen table (Section 3.3) and its offline builder (Section 4.1): a corpus counted by hand,
+"""Pins for the oracle's frozen table (Section 3.3) and its offline builder (Section 4): a corpus counted by hand,
 counts re-derived with vectorised window comparisons and numpy's bincount, a dual-table draft worked by hand, and the
 special cases in which the dual draft must reduce to the single-table one."""
 import numpy as np

@@ -58,7 +58,7 @@ CONFIGS["c1_evict256"] = replace(CONFIGS["c1_tiny"], name="c1_evict256", LC=256)
 CONFIGS["c1_evict1024"] = replace(CONFIGS["c1_tiny"], name="c1_evict1024", LC=1024)
 CONFIGS["c3_evict256"] = replace(CONFIGS["c3_8b_gqa"], name="c3_evict256", LC=256, batch=4)
 CONFIGS["c3_evict1024"] = replace(CONFIGS["c3_8b_gqa"], name="c3_evict1024", LC=1024, batch=4)
-# The paper's tuned table regime (Section 4.1: LL = 1, LC = 2^20, FL = 3, FC = 128, TDL = 96, CRT = 16) on config 2's model
+# The paper's tuned table regime (Section 4: LL = 1, LC = 2^20, FL = 3, FC = 128, TDL = 96, CRT = 16) on config 2's model
 # shape; the depth cap (8 followers deep) is a choice made here.  The second variant shrinks the capacities so that both
 # LRU domains evict, with a follower capacity that is not a multiple of the warp width.
 CONFIGS["p_tuned"] = replace(CONFIGS["c2_7b"], name="p_tuned", LL=1, FL=3, LC=1 << 20, FC=128, max_nodes=96, crt=16,
