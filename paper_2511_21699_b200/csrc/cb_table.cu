@@ -16,6 +16,9 @@ struct Probe {
 };
 
 // Warp-wide lookup of a leader. mykey = key[lane] for lane < LL (0 otherwise), identical call in all lanes.
+// SHARED: other SMs publish index words and entries while this warp probes (bulk update), so index and key are read
+// through to L2 instead of from an L1 line that may be stale.
+template <bool SHARED = false>
 __device__ __forceinline__ Probe tbl_find(const CbTables& t, const CbSeq& s, int32_t mykey, uint64_t h, int lane) {
     Probe r;
     r.eid = -2; r.slot = 0; r.free_slot = 0xFFFFFFFFu; r.probes = 0;
@@ -23,15 +26,17 @@ __device__ __forceinline__ Probe tbl_find(const CbTables& t, const CbSeq& s, int
     uint32_t bucket = cb_hash_bucket(h, t.nslots);
     for (uint32_t p = 0; p < nb; ++p) {
         r.probes = p + 1;
-        // read through to L2: in the bulk update other SMs publish index words and entries while this warp probes
-        const uint32_t w = __ldcg(&s.index[bucket * 32 + lane]);
+        const uint32_t w = SHARED ? __ldcg(&s.index[bucket * 32 + lane]) : s.index[bucket * 32 + lane];
         uint32_t cand = __ballot_sync(CB_FULL, w != CB_IDX_EMPTY && w != CB_IDX_TOMB && (w >> CB_EID_BITS) == tag);
         while (cand) {
             const int l = __ffs(cand) - 1;
             cand &= cand - 1;
             const uint32_t eid = __shfl_sync(CB_FULL, w, l) & CB_EID_MASK;
             bool eq = true;
-            if (lane < t.LL) eq = ((int32_t)__ldcg(&s.entries[(size_t)eid * t.E + lane]) == mykey);
+            if (lane < t.LL) {
+                const uint32_t* kp = &s.entries[(size_t)eid * t.E + lane];
+                eq = ((int32_t)(SHARED ? __ldcg(kp) : *kp) == mykey);
+            }
             if (__all_sync(CB_FULL, eq)) { r.eid = (int)eid; r.slot = bucket * 32 + l; return r; }
         }
         const uint32_t fr = __ballot_sync(CB_FULL, w == CB_IDX_EMPTY || w == CB_IDX_TOMB);
@@ -225,7 +230,7 @@ __device__ void tbl_insert_shared(const CbTables& t, const CbSeq& s, int32_t myk
     const uint32_t tagword = cb_hash_tag(h) << CB_EID_BITS;
     int eid = -1;
     for (int attempt = 0; attempt < 64; ++attempt) {            // a claim can lose its slot to another warp's leader: look again
-        const Probe pr = tbl_find(t, s, mykey, h, lane);
+        const Probe pr = tbl_find<true>(t, s, mykey, h, lane);
         cnt.maxprobe = max(cnt.maxprobe, pr.probes);
         if (pr.eid >= 0) {
             uint32_t* e = s.entries + (size_t)pr.eid * t.E;
