@@ -144,6 +144,7 @@ extern "C" cb_status cb_tree_attn(cb_ctx* ctx, const cb_attn_args* a, void* stre
     p.status = ctx->d_status;
     // The tensor-core kernel is persistent: one CTA per SM, each taking an equal share of all key tiles.
     p.nc = ctx->num_sms < CB_ATTN_MAX_CTAS ? ctx->num_sms : CB_ATTN_MAX_CTAS;
+    p.cs = 0;
     cudaStream_t st = (cudaStream_t)stream;
     if (c.flags & CB_FLAG_ATTN_CUDA_CORES) return cb_attn_launch_cuda_cores(ctx, p, st);
     return cb_attn_launch_tensor(ctx, p, st);

@@ -33,6 +33,7 @@ struct CbAttnParams {
     int NPT;              // tree nodes per row tile = 128 / G
     int MT;               // row tiles that T nodes need = ceil(T / NPT)
     int nc;               // persistent CTAs (= ranges of the global tile sequence)
+    int cs;               // > 0: cluster mode, one unit per cluster of cs CTAs (see cb_attn_tc.cu); 0: the stream-K split
     float scale_log2;     // softmax scale * log2(e)
     uint32_t* status;
 };
@@ -110,11 +111,22 @@ struct CbWalker {
     long long g, g1, pre;
     int b;
     CbSeqShape s;
+    bool fixed, fixed_left;   // cluster mode: the CTA has exactly one share of one unit (or none)
+    CbUnit fu;
     __device__ __forceinline__ void init(const CbAttnParams& p, long long g0, long long g1_, int b0, long long pre0) {
-        g = g0; g1 = g1_; b = b0; pre = pre0;
+        g = g0; g1 = g1_; b = b0; pre = pre0; fixed = false; fixed_left = false;
         if (g < g1) s = cb_seq_shape(p, b);
     }
+    __device__ __forceinline__ void init_fixed(const CbUnit& u0) {
+        g = 0; g1 = 0; b = 0; pre = 0; fixed = true; fixed_left = u0.t1 > u0.t0; fu = u0;
+    }
     __device__ __forceinline__ bool next(const CbAttnParams& p, CbUnit* u) {
+        if (fixed) {
+            if (!fixed_left) return false;
+            fixed_left = false;
+            *u = fu;
+            return true;
+        }
         while (true) {
             if (g >= g1) return false;
             while (g >= pre + s.W) { pre += s.W; ++b; s = cb_seq_shape(p, b); }

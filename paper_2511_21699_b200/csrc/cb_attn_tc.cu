@@ -70,6 +70,41 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
+// Cluster-scope helpers: address of a shared-memory location in another CTA of the cluster, arrival on a barrier there
+// (releasing this thread's earlier writes to the cluster), a 16-byte store there, and a bounded wait that acquires them.
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t local, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+__device__ __forceinline__ void st_cluster_v4(uint32_t raddr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(raddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
+    return ok;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
+    if (mbar_try_cluster(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        if (mbar_try_cluster(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) break;
+    }
+    *abort_flag = 1;
+    atomicCAS(status, 0u, (uint32_t)CB_ERR_TIMEOUT);
+    return false;
+}
+
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
@@ -216,15 +251,16 @@ struct Cfg {
     static constexpr uint32_t OFF_Q = 0;                     // two row tiles
     static constexpr uint32_t OFF_RING = 2 * Q_BYTES;
     static constexpr uint32_t OFF_BAR = OFF_RING + NSLOT * TILE_BYTES;
-    // slot_full[NSLOT], slot_free[NSLOT], q_full, q_free, s_full0, p_ready[2], o_free[2]
-    static constexpr int NBAR = 2 * NSLOT + 2 + 5;
+    // slot_full[NSLOT], slot_free[NSLOT], q_full, q_free, s_full0, p_ready[2], o_free[2], cluster_ready, cluster_data
+    static constexpr int NBAR = 2 * NSLOT + 2 + 7;
     static constexpr uint32_t OFF_MISC = OFF_BAR + NBAR * 8;  // schedule, tmem base, abort flag
-    static constexpr uint32_t SMEM = OFF_MISC + 64;
+    static constexpr uint32_t SMEM = OFF_MISC + 96;
     static constexpr uint32_t SMEM_ALLOC = SMEM + 1024;      // slack to align the base to 1024 bytes
     static constexpr uint32_t O_COL = 256;                   // TMEM columns: S0 at 0, S1 at 128, O0 at 256, O1 at 256 + D
 };
 
-struct SchedSmem { long long g0, g1, pre0; int b0; };
+struct SchedSmem { long long g0, g1, pre0; int b0; int c_b, c_kh, c_t0, c_t1, c_tiles, c_n, c_ctx, c_has; };
+static_assert(sizeof(SchedSmem) <= 64, "the schedule block is followed by the tmem base and the abort flag");
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -245,9 +281,10 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     const uint32_t bar_sfull0 = bar0 + 8u * (2 * C::NSLOT + 2);
     auto bar_pready = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 3 + s); };
     auto bar_ofree = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 5 + s); };
+    const uint32_t bar_cready = bar0 + 8u * (2 * C::NSLOT + 7), bar_cdata = bar_cready + 8u;   // cluster mode only
     SchedSmem* s_sched = reinterpret_cast<SchedSmem*>(sgen + C::OFF_MISC);
-    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sgen + C::OFF_MISC + 32);
-    volatile int* s_abort = reinterpret_cast<volatile int*>(sgen + C::OFF_MISC + 36);
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sgen + C::OFF_MISC + 64);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(sgen + C::OFF_MISC + 68);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
@@ -266,6 +303,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             for (int s = 0; s < 2; ++s) {
                 mbar_init(bar_pready(s), 128); mbar_init(bar_ofree(s), 128);
             }
+            mbar_init(bar_cready, p.cs > 0 ? (uint32_t)p.cs : 1u); mbar_init(bar_cdata, 128);
             *s_abort = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             tma_prefetch_desc(&maps.k_pool); tma_prefetch_desc(&maps.v_pool); tma_prefetch_desc(&maps.q);
@@ -274,7 +312,19 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     }
     CB_PDL_ENTRY();
 
-    if (warp == 0) {
+    if (warp == 0 && p.cs > 0) {
+        // Cluster mode: cluster k works on unit k = (sequence, kv head) and its CTAs take equal parts of the unit's key tiles.
+        if (lane == 0) {
+            const int uid = cta / p.cs, rank = cta % p.cs;
+            const int b = uid / p.Hkv;
+            const CbSeqShape sh = cb_seq_shape(p, b);
+            s_sched->c_b = b; s_sched->c_kh = uid % p.Hkv; s_sched->c_tiles = sh.tiles; s_sched->c_n = sh.n; s_sched->c_ctx = sh.ctx;
+            s_sched->c_has = sh.RG > 0 ? 1 : 0;
+            s_sched->c_t0 = sh.RG > 0 ? (int)((long long)sh.tiles * rank / p.cs) : 0;
+            s_sched->c_t1 = sh.RG > 0 ? (int)((long long)sh.tiles * (rank + 1) / p.cs) : 0;
+            s_sched->g0 = 0; s_sched->g1 = 0; s_sched->pre0 = 0; s_sched->b0 = 0;
+        }
+    } else if (warp == 0) {
         // this CTA's range of the global tile sequence
         const long long tot = cb_sched_total(p, lane);
         const long long g0 = cb_range_start(tot, p.nc, cta), g1 = cb_range_start(tot, p.nc, cta + 1);
@@ -290,7 +340,17 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     const long long g0 = s_sched->g0, g1 = s_sched->g1, pre0 = s_sched->pre0;
     const int b0 = s_sched->b0;
     CbWalker wk;
-    wk.init(p, g0, g1, b0, pre0);
+    if (p.cs > 0) {
+        // the peers' barriers must exist before anything arrives on them
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        CbUnit u0;
+        u0.b = s_sched->c_b; u0.kh = s_sched->c_kh; u0.rg = 0; u0.t0 = s_sched->c_t0; u0.t1 = s_sched->c_t1;
+        u0.tiles = s_sched->c_tiles; u0.n = s_sched->c_n; u0.ctx = s_sched->c_ctx; u0.nrt = 1;
+        wk.init_fixed(u0);
+    } else {
+        wk.init(p, g0, g1, b0, pre0);
+    }
     CbUnit u;
 
     if (warp < 4) {
@@ -469,6 +529,8 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             }
             return have;
         };
+        float c_m = -INFINITY, c_l = 0.f;                     // cluster mode: this CTA's share of the unit, kept for the exchange
+        bool c_share = false;
         bool have = fetch_next();
         while (ok && have) {
             u = un;
@@ -610,7 +672,9 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             // ---- epilogue of this unit's share: O is complete once its last PV has finished
             if (!(ok = wait_pv(u.t1 - 1))) break;
             tc_fence_after();
-            if (warp_active) {
+            if (p.cs > 0) {
+                c_m = m_used; c_l = l; c_share = true;         // O stays in TMEM until the exchange below
+            } else if (warp_active) {
                 const bool whole = u.t0 == 0 && u.t1 == u.tiles;
                 if (whole) {
                     const float inv = l > 0.f ? 1.0f / l : 0.f;
@@ -650,6 +714,85 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             }
             tc_fence_before();
             mbar_arrive(bar_ofree(wg));
+        }
+        if (p.cs > 0 && s_sched->c_has) {
+            // ------------------------------------------------------------------ cluster mode: combine the unit's shares
+            // Every CTA of the cluster holds the unnormalised rows of its share (O in TMEM, running maximum and sum in
+            // registers).  Row block r (128 / cs rows) is combined by CTA r: each CTA writes its rows of block r into that
+            // CTA's shared memory (over the K/V ring, which is idle once all CTAs have reported their last product done),
+            // arrives on its barrier, and the owner merges the cs contributions and writes the output rows.
+            const int cs = p.cs, R = CB_MT / cs, rank = cta % cs;
+            const int cb_ = s_sched->c_b, ckh = s_sched->c_kh, cn = s_sched->c_n;
+            const uint32_t recv = sbase + C::OFF_RING;        // [cs sources][R rows][D + 4] floats
+            constexpr uint32_t ROWB = (D + 4) * 4;
+            if (ok && wg == 0 && row == 0)
+                for (int r = 0; r < cs; ++r) mbar_arrive_remote(cluster_addr(bar_cready, (uint32_t)r));
+            if (ok) ok = mbar_wait_cluster(bar_cready, 0, s_abort, p.status);
+            if (ok && wg == 0) {
+                const int dest = row / R, rl = row % R;
+                const bool valid = row < RT && (row / p.G) < cn;
+                const uint32_t ra = cluster_addr(recv + (uint32_t)(rank * R + rl) * ROWB, (uint32_t)dest);
+                const bool act = (wq * 32) < RT && ((wq * 32) / p.G) < cn;     // row 0 of the warp is valid
+                if (act && c_share) {
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        CB_TMEM_LD32(o, 0, tm_O + c * 32);
+                        tmem_wait_ld();
+                        if (valid) {
+#pragma unroll
+                            for (int v4 = 0; v4 < 8; ++v4)
+                                st_cluster_v4(ra + (uint32_t)(c * 32 + v4 * 4) * 4u, o[v4 * 4], o[v4 * 4 + 1], o[v4 * 4 + 2], o[v4 * 4 + 3]);
+                        }
+                    }
+                }
+                if (valid) st_cluster_v4(ra + D * 4u, __float_as_uint(c_share ? c_m : -INFINITY), __float_as_uint(c_share ? c_l : 0.f), 0u, 0u);
+                mbar_arrive_remote(cluster_addr(bar_cdata, (uint32_t)dest));
+            }
+            if (ok) ok = mbar_wait_cluster(bar_cdata, 0, s_abort, p.status);
+            if (ok) {
+                // 256 threads: 256 / R threads per row, each a run of D * R / 256 columns in groups of 8
+                const int t = wg * 128 + row, tpr = 256 / R, rl = t / tpr, sub = t % tpr;
+                const int gr = rank * R + rl, node = gr / p.G, h = ckh * p.G + gr % p.G;
+                if (gr < RT && node < cn) {
+                    float mx = -INFINITY;
+                    for (int sidx = 0; sidx < cs; ++sidx) {
+                        float ms;
+                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(ms) : "r"(recv + (uint32_t)(sidx * R + rl) * ROWB + D * 4u));
+                        mx = fmaxf(mx, ms);
+                    }
+                    float wsum = 0.f;
+                    for (int sidx = 0; sidx < cs; ++sidx) {
+                        float ms, ls;
+                        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(ms), "=f"(ls) : "r"(recv + (uint32_t)(sidx * R + rl) * ROWB + D * 4u));
+                        wsum += (ms == -INFINITY) ? 0.f : ex2(ms - mx) * ls;
+                    }
+                    const float inv = wsum > 0.f ? 1.0f / wsum : 0.f;
+                    const int cols = D / tpr;
+                    for (int g8 = 0; g8 < cols; g8 += 8) {
+                        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                        for (int sidx = 0; sidx < cs; ++sidx) {
+                            const uint32_t base = recv + (uint32_t)(sidx * R + rl) * ROWB;
+                            float ms;
+                            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(ms) : "r"(base + D * 4u));
+                            if (ms == -INFINITY) continue;      // that CTA had no tiles: its row was not written
+                            const float w = ex2(ms - mx);
+                            float v[8];
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3])
+                                         : "r"(base + (uint32_t)(sub * cols + g8) * 4u));
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                                         : "r"(base + (uint32_t)(sub * cols + g8 + 4) * 4u));
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) acc[k] += w * v[k];
+                        }
+                        __nv_bfloat16* op = p.out + (((size_t)cb_ * p.T + node) * p.Hq + h) * D + sub * cols + g8;
+                        *reinterpret_cast<uint4*>(op) = make_uint4(pack_bf16(acc[0] * inv, acc[1] * inv), pack_bf16(acc[2] * inv, acc[3] * inv),
+                                                                   pack_bf16(acc[4] * inv, acc[5] * inv), pack_bf16(acc[6] * inv, acc[7] * inv));
+                    }
+                    if (sub == 0 && p.lse)
+                        p.lse[((size_t)cb_ * p.Hq + h) * p.T + node] = wsum > 0.f ? (mx + log2f(wsum)) * 0.6931471805599453f : 0.f;
+                }
+            }
         }
     }
 
@@ -783,12 +926,54 @@ bool encode_map(CUtensorMap* m, const void* base, int D, int heads, int rows, lo
     return r == CUDA_SUCCESS;
 }
 
+// Cluster mode is for launches with few units, where the stream-K split would make every unit a shared one: all trees fit
+// one row tile (so a unit is one (sequence, kv head)) and the units times a cluster size of 8, 4 or 2 fill at least 60% of
+// the SMs without exceeding them, and that many clusters can be resident at once.  Returns the cluster size or 0.
 template <int D>
-cb_status launch(const CbAttnParams& p, const TcMaps& maps, cudaStream_t st) {
+int pick_cluster_size(const CbAttnParams& p, int num_sms) {
+    if (p.MT != 1) return 0;
+    const long long units = (long long)p.B * p.Hkv;
+    for (int cs = 8; cs >= 2; cs >>= 1) {
+        if (units * cs > num_sms || units * cs * 10 < (long long)num_sms * 6) continue;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(units * cs)); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = Cfg<D>::SMEM_ALLOC;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = (unsigned)cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        int nclusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&nclusters, cb_attn_tc_kernel<D>, &cfg) != cudaSuccess) { (void)cudaGetLastError(); continue; }
+        if (nclusters >= units) return cs;
+    }
+    return 0;
+}
+
+template <int D>
+cb_status launch(CbAttnParams p, const TcMaps& maps, cudaStream_t st, int num_sms) {
     static bool attr_set = false;
     if (!attr_set) {
         CB_CUDA(cudaFuncSetAttribute(cb_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<D>::SMEM_ALLOC));
         attr_set = true;
+    }
+    // the choice depends on the shape only: remember it for the shapes seen last
+    static int memo_key[4] = {-1, -1, -1, -1}, memo_cs = 0;
+    if (memo_key[0] != p.B || memo_key[1] != p.Hkv || memo_key[2] != p.MT || memo_key[3] != num_sms) {
+        memo_cs = pick_cluster_size<D>(p, num_sms);
+        memo_key[0] = p.B; memo_key[1] = p.Hkv; memo_key[2] = p.MT; memo_key[3] = num_sms;
+    }
+    p.cs = memo_cs;
+    if (p.cs > 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(p.B * p.Hkv * p.cs)); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = Cfg<D>::SMEM_ALLOC; cfg.stream = st;
+        cudaLaunchAttribute at[2];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = (unsigned)p.cs; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at; cfg.numAttrs = 2;
+        CB_CUDA(cudaLaunchKernelEx(&cfg, cb_attn_tc_kernel<D>, p, maps));
+        cb_count_launch(1);
+        return CB_OK;
     }
     CB_CUDA(cb_launch_pdl(cb_attn_tc_kernel<D>, dim3(p.nc), dim3(kThreads), Cfg<D>::SMEM_ALLOC, st, p, maps));
     CB_CUDA(cb_launch_pdl(cb_attn_merge_kernel<D>, dim3(p.nc, 4), dim3(256), 0, st, p));
@@ -818,7 +1003,6 @@ std::mutex g_map_mutex;
 }  // namespace
 
 cb_status cb_attn_launch_tensor(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t st) {
-    (void)ctx;
     if (p.P != 16) return CB_ERR_UNSUPPORTED;
     const MapKey key = {p.q, p.k_pool, p.v_pool, p.k_tree, p.v_tree, p.D, p.Hq, p.Hkv, p.P, p.T, p.B, p.G, p.NPT, p.num_pages};
     TcMaps maps;
@@ -839,5 +1023,5 @@ cb_status cb_attn_launch_tensor(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t
         g_map_keys[slot] = key;
         g_map_vals[slot] = maps;
     }
-    return p.D == 128 ? launch<128>(p, maps, st) : launch<64>(p, maps, st);
+    return p.D == 128 ? launch<128>(p, maps, st, ctx->num_sms) : launch<64>(p, maps, st, ctx->num_sms);
 }
