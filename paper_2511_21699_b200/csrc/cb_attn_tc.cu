@@ -18,6 +18,11 @@
 // the tensor pipe works on one tile's MMAs while the other tile is in softmax).  A unit with one valid
 // row tile is handled by warpgroup 0 alone with S double-buffered over S0/S1.
 // All waits are bounded; a wait that runs out records CB_ERR_TIMEOUT and the CTA drains and exits.
+//
+// Cluster mode.  When a launch has so few units that the split above would make every unit a shared one (batch 1), the
+// kernel is launched as thread-block clusters instead: cluster k works on unit k, its CTAs take equal parts of the unit's
+// key tiles, and at the end they combine their shares through distributed shared memory: row block r of the 128 rows is
+// gathered in CTA r, which merges the contributions and writes the output.  No partials go to HBM and no merge pass runs.
 #include <cuda.h>
 
 #include <mutex>
