@@ -756,10 +756,10 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             }
             if (ok) ok = mbar_wait_cluster(bar_cdata, 0, s_abort, p.status);
             if (ok) {
-                // 256 threads: 256 / R threads per row, each a run of D * R / 256 columns in groups of 8
-                const int t = wg * 128 + row, tpr = 256 / R, rl = t / tpr, sub = t % tpr;
+                // up to 256 threads: tpr threads per row, each a run of D / tpr >= 8 columns in groups of 8
+                const int t = wg * 128 + row, tpr = min(256 / R, D / 8), rl = t / tpr, sub = t % tpr;
                 const int gr = rank * R + rl, node = gr / p.G, h = ckh * p.G + gr % p.G;
-                if (gr < RT && node < cn) {
+                if (rl < R && gr < RT && node < cn) {
                     float mx = -INFINITY;
                     for (int sidx = 0; sidx < cs; ++sidx) {
                         float ms;

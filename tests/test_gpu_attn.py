@@ -85,6 +85,36 @@ def test_attn_ragged_contexts_gqa(oracle, flags):
     _run(SMALL_GQA, oracle, False, _all, flags=flags, ctx_override=[0, 1, 16, 256, 299])
 
 
+# Few units: the kernel runs as thread-block clusters, one unit per cluster (32 heads x 4 CTAs, 2 x 32 heads x 2 CTAs,
+# 16 kv heads x 8 CTAs with head_dim 64).  Contexts shorter than the cluster (some CTAs get no key tile), ragged ones, none.
+CLUSTER_4 = W.CbConfig("cluster4", 1, 2, 2, 64, 2, 40, 6, 0, 32, 32, 128, (0, 700), 100, 1.1, 0.3, (4, 8), 64)
+CLUSTER_2 = W.CbConfig("cluster2", 2, 2, 2, 64, 2, 64, 6, 0, 32, 32, 128, (0, 700), 100, 1.1, 0.3, (4, 8), 64)
+CLUSTER_8 = W.CbConfig("cluster8", 1, 2, 2, 64, 2, 24, 6, 0, 64, 16, 64, (0, 700), 100, 1.1, 0.3, (4, 8), 64)
+
+
+@pytest.mark.parametrize("cfg,ctxs", [(CLUSTER_4, [[0], [1], [129], [600]]), (CLUSTER_2, [[0, 299], [385, 16]]),
+                                      (CLUSTER_8, [[0], [257], [700]])])
+def test_attn_cluster_mode_ragged(oracle, cfg, ctxs):
+    for ctx in ctxs:
+        _run(cfg, oracle, False, _sampled(2, 4, 8), ctx_override=ctx)
+
+
+def test_attn_cluster_mode_empty_tree(oracle):
+    """A batch of one whose tree is empty: every output row is padding."""
+    from paper_2511_21699_b200 import Cacheback
+    cfg = CLUSTER_4
+    prob = Problem(cfg)
+    d = device_attn_inputs(cfg, prob)
+    cb = Cacheback.from_config(cfg)
+    T = cfg.max_nodes
+    out = torch.full((1, T, cfg.n_q_heads, cfg.head_dim), 3.0, dtype=torch.bfloat16, device="cuda")
+    mask = torch.zeros((1, T, (T + 31) // 32), dtype=torch.int32, device="cuda")
+    cb.cb_tree_attn(d["q"], d["k_pool"], d["v_pool"], d["block_table"], d["ctx_len"], d["k_tree"], d["v_tree"], mask,
+                    torch.zeros(1, dtype=torch.int32, device="cuda"), out=out)
+    torch.cuda.synchronize()
+    assert cb.cb_poll_status()[0] == 0 and (out == 0).all()
+
+
 @pytest.mark.parametrize("name", ["c2_7b", "c3_8b_gqa", "c4_13b_turns", "p_tuned"])
 @pytest.mark.parametrize("full", [True, False])
 def test_attn_full_size_sampled(oracle, name, full):
