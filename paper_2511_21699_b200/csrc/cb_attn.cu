@@ -145,6 +145,11 @@ extern "C" cb_status cb_tree_attn(cb_ctx* ctx, const cb_attn_args* a, void* stre
     // The tensor-core kernel is persistent: one CTA per SM, each taking an equal share of all key tiles.
     p.nc = ctx->num_sms < CB_ATTN_MAX_CTAS ? ctx->num_sms : CB_ATTN_MAX_CTAS;
     p.cs = 0;
+    {
+        const long long cap = (long long)a->max_pages * c.page_size;
+        const long long mc = a->max_ctx > 0 && a->max_ctx < cap ? a->max_ctx : cap;
+        p.max_tiles = (int)((mc + CB_KT - 1) / CB_KT) + 1;
+    }
     cudaStream_t st = (cudaStream_t)stream;
     if (c.flags & CB_FLAG_ATTN_CUDA_CORES) return cb_attn_launch_cuda_cores(ctx, p, st);
     return cb_attn_launch_tensor(ctx, p, st);

@@ -33,6 +33,7 @@ struct CbAttnParams {
     int NPT;              // tree nodes per row tile = 128 / G
     int MT;               // row tiles that T nodes need = ceil(T / NPT)
     int nc;               // persistent CTAs (= ranges of the global tile sequence)
+    int max_tiles;        // host's upper bound on the key tiles of a unit (from max_ctx, else from the block table's width)
     int cs;               // > 0: cluster mode, one unit per cluster of cs CTAs (see cb_attn_tc.cu); 0: the stream-K split
     float scale_log2;     // softmax scale * log2(e)
     uint32_t* status;

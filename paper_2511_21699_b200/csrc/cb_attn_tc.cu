@@ -932,14 +932,17 @@ bool encode_map(CUtensorMap* m, const void* base, int D, int heads, int rows, lo
 }
 
 // Cluster mode is for launches with few units, where the stream-K split would make every unit a shared one: all trees fit
-// one row tile (so a unit is one (sequence, kv head)) and the units times a cluster size of 8, 4 or 2 fill at least 60% of
-// the SMs without exceeding them, and that many clusters can be resident at once.  Returns the cluster size or 0.
+// one row tile (so a unit is one (sequence, kv head)), units times a cluster size of 8, 4 or 2 does not exceed the SMs, that
+// many clusters can be resident at once, and a CTA's part of a unit (tiles / cs) is shorter than a CTA's range under the
+// stream-K split plus what its partials and merge pass cost (about three tiles).  Returns the cluster size or 0.
 template <int D>
 int pick_cluster_size(const CbAttnParams& p, int num_sms) {
     if (p.MT != 1) return 0;
     const long long units = (long long)p.B * p.Hkv;
     for (int cs = 8; cs >= 2; cs >>= 1) {
-        if (units * cs > num_sms || units * cs * 10 < (long long)num_sms * 6) continue;
+        if (units * cs > num_sms) continue;
+        const long long in_cluster = (p.max_tiles + cs - 1) / cs, stream_k = units * (p.max_tiles + 2) / num_sms + 3;
+        if (in_cluster >= stream_k) continue;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(units * cs)); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = Cfg<D>::SMEM_ALLOC;
         cudaLaunchAttribute at[1];
@@ -961,10 +964,10 @@ cb_status launch(CbAttnParams p, const TcMaps& maps, cudaStream_t st, int num_sm
         attr_set = true;
     }
     // the choice depends on the shape only: remember it for the shapes seen last
-    static int memo_key[4] = {-1, -1, -1, -1}, memo_cs = 0;
-    if (memo_key[0] != p.B || memo_key[1] != p.Hkv || memo_key[2] != p.MT || memo_key[3] != num_sms) {
+    static int memo_key[5] = {-1, -1, -1, -1, -1}, memo_cs = 0;
+    if (memo_key[0] != p.B || memo_key[1] != p.Hkv || memo_key[2] != p.MT || memo_key[3] != num_sms || memo_key[4] != p.max_tiles) {
         memo_cs = pick_cluster_size<D>(p, num_sms);
-        memo_key[0] = p.B; memo_key[1] = p.Hkv; memo_key[2] = p.MT; memo_key[3] = num_sms;
+        memo_key[0] = p.B; memo_key[1] = p.Hkv; memo_key[2] = p.MT; memo_key[3] = num_sms; memo_key[4] = p.max_tiles;
     }
     p.cs = memo_cs;
     if (p.cs > 0) {
