@@ -490,6 +490,15 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                                         (u.rg * 2 + rt) * p.NPT, u.b);
                     ++uq;
                 }
+                if (p.cs > 0 && s_sched->c_has) {
+                    // Cluster mode: the peers write their rows into this CTA's query tiles, so it reports itself ready to
+                    // receive as soon as its last S product has released them (long before its last P.V is done).
+                    const int Rv = (min(RT, p.T * p.G) + p.cs - 1) / p.cs;
+                    if ((uint32_t)(p.cs * Rv) * (uint32_t)((D + 4) * 4) <= 2u * C::Q_BYTES) {
+                        if (uq == 0 || mbar_wait(bar_qfree, 0, s_abort, p.status))
+                            for (int r = 0; r < p.cs; ++r) mbar_arrive_remote(cluster_addr(bar_cready, (uint32_t)r));
+                    }
+                }
             }
             __syncwarp();
         } else {
@@ -723,20 +732,23 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
         if (p.cs > 0 && s_sched->c_has) {
             // ------------------------------------------------------------------ cluster mode: combine the unit's shares
             // Every CTA of the cluster holds the unnormalised rows of its share (O in TMEM, running maximum and sum in
-            // registers).  Row block r (128 / cs rows) is combined by CTA r: each CTA writes its rows of block r into that
-            // CTA's shared memory (over the K/V ring, which is idle once all CTAs have reported their last product done),
-            // arrives on its barrier, and the owner merges the cs contributions and writes the output rows.
-            const int cs = p.cs, R = CB_MT / cs, rank = cta % cs;
+            // registers).  Row i is combined by CTA i % cs: each CTA writes its copy of the row into that CTA's shared memory,
+            // arrives on its data barrier, and the owner merges the cs contributions and writes the output row.  The rows are
+            // received in the two query tiles when they fit (they are idle from a CTA's last S product on, which the query
+            // loader reports), otherwise in the K/V ring (idle from the last P.V on, reported here).
+            const int cs = p.cs, rank = cta % cs;
+            const int Rv = (min(RT, p.T * p.G) + cs - 1) / cs;   // rows that one CTA may own (rows beyond T nodes never exist)
             const int cb_ = s_sched->c_b, ckh = s_sched->c_kh, cn = s_sched->c_n;
-            const uint32_t recv = sbase + C::OFF_RING;        // [cs sources][R rows][D + 4] floats
             constexpr uint32_t ROWB = (D + 4) * 4;
-            if (ok && wg == 0 && row == 0)
+            const bool in_q = (uint32_t)(cs * Rv) * ROWB <= 2u * C::Q_BYTES;
+            const uint32_t recv = sbase + (in_q ? C::OFF_Q : C::OFF_RING);     // [cs sources][Rv rows][D + 4] floats
+            if (ok && !in_q && wg == 0 && row == 0)
                 for (int r = 0; r < cs; ++r) mbar_arrive_remote(cluster_addr(bar_cready, (uint32_t)r));
             if (ok) ok = mbar_wait_cluster(bar_cready, 0, s_abort, p.status);
             if (ok && wg == 0) {
-                const int dest = row / R, rl = row % R;
+                const int dest = row % cs, rl = row / cs;
                 const bool valid = row < RT && (row / p.G) < cn;
-                const uint32_t ra = cluster_addr(recv + (uint32_t)(rank * R + rl) * ROWB, (uint32_t)dest);
+                const uint32_t ra = cluster_addr(recv + (uint32_t)(rank * Rv + rl) * ROWB, (uint32_t)dest);
                 const bool act = (wq * 32) < RT && ((wq * 32) / p.G) < cn;     // row 0 of the warp is valid
                 if (act && c_share) {
 #pragma unroll
@@ -757,19 +769,21 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             if (ok) ok = mbar_wait_cluster(bar_cdata, 0, s_abort, p.status);
             if (ok) {
                 // up to 256 threads: tpr threads per row, each a run of D / tpr >= 8 columns in groups of 8
-                const int t = wg * 128 + row, tpr = min(256 / R, D / 8), rl = t / tpr, sub = t % tpr;
-                const int gr = rank * R + rl, node = gr / p.G, h = ckh * p.G + gr % p.G;
-                if (rl < R && gr < RT && node < cn) {
+                int tpr = D / 8;                                 // a power of two
+                while (tpr * Rv > 256) tpr >>= 1;
+                const int t = wg * 128 + row, rl = t / tpr, sub = t % tpr;
+                const int gr = rl * cs + rank, node = gr / p.G, h = ckh * p.G + gr % p.G;
+                if (rl < Rv && gr < RT && node < cn) {
                     float mx = -INFINITY;
                     for (int sidx = 0; sidx < cs; ++sidx) {
                         float ms;
-                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(ms) : "r"(recv + (uint32_t)(sidx * R + rl) * ROWB + D * 4u));
+                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(ms) : "r"(recv + (uint32_t)(sidx * Rv + rl) * ROWB + D * 4u));
                         mx = fmaxf(mx, ms);
                     }
                     float wsum = 0.f;
                     for (int sidx = 0; sidx < cs; ++sidx) {
                         float ms, ls;
-                        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(ms), "=f"(ls) : "r"(recv + (uint32_t)(sidx * R + rl) * ROWB + D * 4u));
+                        asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(ms), "=f"(ls) : "r"(recv + (uint32_t)(sidx * Rv + rl) * ROWB + D * 4u));
                         wsum += (ms == -INFINITY) ? 0.f : ex2(ms - mx) * ls;
                     }
                     const float inv = wsum > 0.f ? 1.0f / wsum : 0.f;
@@ -777,7 +791,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     for (int g8 = 0; g8 < cols; g8 += 8) {
                         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
                         for (int sidx = 0; sidx < cs; ++sidx) {
-                            const uint32_t base = recv + (uint32_t)(sidx * R + rl) * ROWB;
+                            const uint32_t base = recv + (uint32_t)(sidx * Rv + rl) * ROWB;
                             float ms;
                             asm volatile("ld.shared.f32 %0, [%1];" : "=f"(ms) : "r"(base + D * 4u));
                             if (ms == -INFINITY) continue;      // that CTA had no tiles: its row was not written
