@@ -36,3 +36,18 @@ def test_host_side_argument_checks_need_no_gpu():
     assert lib.cb_workspace_bytes(ctypes.byref(bad), ctypes.byref(n)) == 1
     assert lib.cb_status_str(4).decode().startswith("hash probe")
     assert lib.cb_accept_static(4096, 16, 4, 100, 1, 1, 1, 1, 8, 0, 100, 1, 1, 1, None, None) == _lib.CB_ERR_STATIC_LIMIT
+
+
+def test_frozen_table_sizes_and_argument_checks_need_no_gpu():
+    from paper_2511_21699_b200 import _lib
+    lib = _lib.load()
+    n, m = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    cfg = _lib.CbFrozenConfigC(1, 3, 1 << 16, 128)
+    assert lib.cb_frozen_bytes(ctypes.byref(cfg), ctypes.byref(n)) == 0
+    assert n.value >= (1 << 16) * (1 + 128 * 4) * 4                               # entries: key + FC * (stamp + FL tokens)
+    assert lib.cb_frozen_build_bytes(ctypes.byref(cfg), 1 << 20, ctypes.byref(m)) == 0 and m.value > (1 << 20) * 32
+    assert lib.cb_frozen_build_bytes(ctypes.byref(cfg), (1 << 30) + 1, ctypes.byref(m)) == 1   # corpus above the stated limit
+    for bad in (_lib.CbFrozenConfigC(0, 3, 16, 4), _lib.CbFrozenConfigC(1, 9, 16, 4), _lib.CbFrozenConfigC(1, 3, 16, 129),
+                _lib.CbFrozenConfigC(1, 3, (1 << 20) + 1, 4)):
+        assert lib.cb_frozen_bytes(ctypes.byref(bad), ctypes.byref(n)) == 1
+    assert lib.cb_frozen_attach(None, ctypes.byref(cfg), None, 0) == 1            # no context
