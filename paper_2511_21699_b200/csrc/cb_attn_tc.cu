@@ -937,7 +937,10 @@ bool encode_map(CUtensorMap* m, const void* base, int D, int heads, int rows, lo
     cuuint32_t box[4] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           // a head's row is D * 2 bytes contiguous and is fetched as 128-byte halves by two boxes: with D = 128 let the
+                           // first one bring the whole row into L2
+                           D >= 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
         fprintf(stderr, "cacheback: tensor map encode failed (%d): D=%d heads=%d rows=%d blocks=%ld base=%p\n", (int)r, D, heads, rows,
