@@ -18,8 +18,14 @@ struct Probe {
 // Warp-wide lookup of a leader. mykey = key[lane] for lane < LL (0 otherwise), identical call in all lanes.
 // SHARED: other SMs publish index words and entries while this warp probes (bulk update), so index and key are read
 // through to L2 instead of from an L1 line that may be stale.
-template <bool SHARED = false>
-__device__ __forceinline__ Probe tbl_find(const CbTables& t, const CbSeq& s, int32_t mykey, uint64_t h, int lane) {
+// FETCH (tables with FC <= 32, so that lane l owns follower l alone): the follower's stamp and tokens are loaded together
+// with the key when an index word's tag matches, which saves the callers two dependent memory round trips.
+struct EntryRegs {
+    uint32_t fs;
+    int32_t tok[CB_MAX_FL];
+};
+template <bool SHARED = false, bool FETCH = false>
+__device__ __forceinline__ Probe tbl_find(const CbTables& t, const CbSeq& s, int32_t mykey, uint64_t h, int lane, EntryRegs* er = nullptr) {
     Probe r;
     r.eid = -2; r.slot = 0; r.free_slot = 0xFFFFFFFFu; r.probes = 0;
     const uint32_t nb = t.nslots >> 5, tag = cb_hash_tag(h);
@@ -33,7 +39,15 @@ __device__ __forceinline__ Probe tbl_find(const CbTables& t, const CbSeq& s, int
             cand &= cand - 1;
             const uint32_t eid = __shfl_sync(CB_FULL, w, l) & CB_EID_MASK;
             bool eq = true;
-            if (lane < t.LL) {
+            if (FETCH) {
+                const uint32_t* e = s.entries + (size_t)eid * t.E;
+                const bool mine = lane < t.FC;
+                const uint32_t kv = lane < t.LL ? e[lane] : 0u;
+                er->fs = mine ? e[t.LL + lane] : 0u;
+#pragma unroll
+                for (int j = 0; j < CB_MAX_FL; ++j) er->tok[j] = (mine && j < t.FL) ? (int32_t)e[t.LL + t.FC + lane * t.FL + j] : -1;
+                if (lane < t.LL) eq = (int32_t)kv == mykey;
+            } else if (lane < t.LL) {
                 const uint32_t* kp = &s.entries[(size_t)eid * t.E + lane];
                 eq = ((int32_t)(SHARED ? __ldcg(kp) : *kp) == mykey);
             }
@@ -92,6 +106,34 @@ struct TblCounters { uint32_t inserts, levict, fevict, maxprobe; };
 
 // Follower list of an existing leader (Section 3.1): a stored copy of the follower is refreshed, otherwise the follower takes
 // the lowest free place or replaces the least recently inserted one.  e = the leader's entry, c = this operation's stamp.
+// The same with the follower's stamp and tokens already in registers (FC <= 32).
+__device__ __forceinline__ void tbl_put_follower_regs(const CbTables& t, uint32_t* e, const EntryRegs& er, int32_t myfol, uint32_t c, int lane,
+                                                      TblCounters& cnt) {
+    const bool mine = lane < t.FC;
+    bool match = mine && er.fs != 0u;
+#pragma unroll
+    for (int j = 0; j < CB_MAX_FL; ++j) {
+        const int32_t fj = __shfl_sync(CB_FULL, myfol, j);
+        if (j < t.FL) match = match && (er.tok[j] == fj);
+    }
+    const uint32_t mm = __ballot_sync(CB_FULL, match);
+    if (mm) {
+        if (t.refresh && lane == 0) e[t.LL + (__ffs(mm) - 1)] = c;
+        return;
+    }
+    const uint32_t freem = __ballot_sync(CB_FULL, mine && er.fs == 0u);
+    int tgt;
+    if (freem) {
+        tgt = __ffs(freem) - 1;
+    } else {
+        const uint32_t g = __reduce_min_sync(CB_FULL, mine ? er.fs : 0xFFFFFFFFu);
+        tgt = __ffs(__ballot_sync(CB_FULL, mine && er.fs == g)) - 1;
+        cnt.fevict++;
+    }
+    if (lane < t.FL) e[t.LL + t.FC + tgt * t.FL + lane] = (uint32_t)myfol;
+    if (lane == 0) e[t.LL + tgt] = c;
+}
+
 __device__ __forceinline__ void tbl_put_follower(const CbTables& t, uint32_t* e, int32_t myfol, uint32_t c, int lane, TblCounters& cnt) {
     // Lane l looks after followers l, l + 32, ...: one pass finds a stored copy of the follower, the lowest free place
     // and the least recently inserted follower.
@@ -124,17 +166,20 @@ __device__ __forceinline__ void tbl_put_follower(const CbTables& t, uint32_t* e,
 }
 
 // One insertion (Section 3.1). mykey = leader[lane] (lane < LL), myfol = follower[lane] (lane < FL).
+template <bool FETCH = false>
 __device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int32_t myfol, uint32_t& clock,
                            uint32_t& count, int lane, uint32_t* status, TblCounters& cnt) {
     const uint32_t c = ++clock;
     cnt.inserts++;
     const uint64_t h = warp_hash(t, mykey);
-    Probe pr = tbl_find(t, s, mykey, h, lane);
+    EntryRegs er;
+    Probe pr = tbl_find<false, FETCH>(t, s, mykey, h, lane, &er);
     cnt.maxprobe = max(cnt.maxprobe, pr.probes);
     if (pr.eid >= 0) {
         uint32_t* e = s.entries + (size_t)pr.eid * t.E;
         if (lane == 0) s.lstamp[pr.eid] = c;
-        tbl_put_follower(t, e, myfol, c, lane, cnt);
+        if (FETCH) tbl_put_follower_regs(t, e, er, myfol, c, lane, cnt);
+        else tbl_put_follower(t, e, myfol, c, lane, cnt);
     } else if (pr.eid == -1) {
         int eid;
         if (count < (uint32_t)t.LC) {
@@ -163,6 +208,7 @@ __device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int
 }
 
 // One warp per sequence; windows are applied in increasing position.
+template <bool FETCH>
 __global__ void __launch_bounds__(128) cb_update_kernel(CbTables t, int B, const int32_t* __restrict__ tokens,
                                                         int64_t row_stride, const int32_t* __restrict__ n_old,
                                                         const int32_t* __restrict__ n_new, uint32_t* status,
@@ -180,7 +226,7 @@ __global__ void __launch_bounds__(128) cb_update_kernel(CbTables t, int B, const
     for (int i = max(0, n0 - w + 1); i + w <= n1; ++i) {
         const int32_t mykey = lane < t.LL ? row[i + lane] : 0;
         const int32_t myfol = lane < t.FL ? row[i + t.LL + lane] : 0;
-        tbl_insert(t, s, mykey, myfol, clock, count, lane, status, cnt);
+        tbl_insert<FETCH>(t, s, mykey, myfol, clock, count, lane, status, cnt);
     }
     if (lane == 0) {
         s.hdr[0] = clock; s.hdr[1] = count;
@@ -338,6 +384,7 @@ struct DraftSmem {
     int32_t* fol;
 };
 
+template <bool FETCH>
 __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, int T, int crt, int max_depth, int NL, int KF,
                                                        const int32_t* __restrict__ tokens, int64_t row_stride,
                                                        const int32_t* __restrict__ seq_len,
@@ -418,7 +465,8 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
                     int eid = -1, nf = 0;
                     if (ok) {
                         const uint64_t h = warp_hash(tt, mykey);
-                        const Probe pr = tbl_find(tt, ss, mykey, h, lane);
+                        EntryRegs er;
+                        const Probe pr = tbl_find<false, FETCH>(tt, ss, mykey, h, lane, &er);
                         if (pr.eid == -2 && lane == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_PROBE_LIMIT);
                         if (pr.eid >= 0) {
                             eid = pr.eid;
@@ -430,7 +478,8 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
                             uint32_t fs[CB_MAX_FC / 32];
 #pragma unroll
                             for (int c = 0; c < CB_MAX_FC / 32; ++c) {
-                                fs[c] = (c * 32 + lane) < tt.FC ? e[tt.LL + c * 32 + lane] : 0u;
+                                if (FETCH) fs[c] = c == 0 ? er.fs : 0u;            // FC <= 32: stamp and tokens came with the lookup
+                                else fs[c] = (c * 32 + lane) < tt.FC ? e[tt.LL + c * 32 + lane] : 0u;
                                 nf += __popc(__ballot_sync(CB_FULL, fs[c] != 0u));
                             }
                             nf = min(nf, min(KF, (leaf == 0 ? max(1, T - crt) : T) - n_now));
@@ -451,8 +500,14 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
                             for (int c = 0; c < CB_MAX_FC / 32; ++c) {
                                 if (rank[c] >= 0) {
                                     const int f = c * 32 + lane;
-                                    for (int j = 0; j < tt.FL; ++j)
-                                        S.fol[li * FLFC + rank[c] * tt.FL + j] = (int32_t)e[tt.LL + tt.FC + f * tt.FL + j];
+                                    if (FETCH) {
+#pragma unroll
+                                        for (int j = 0; j < CB_MAX_FL; ++j)
+                                            if (j < tt.FL) S.fol[li * FLFC + rank[c] * tt.FL + j] = er.tok[j];
+                                    } else {
+                                        for (int j = 0; j < tt.FL; ++j)
+                                            S.fol[li * FLFC + rank[c] * tt.FL + j] = (int32_t)e[tt.LL + tt.FC + f * tt.FL + j];
+                                    }
                                 }
                             }
                         }
@@ -531,7 +586,7 @@ extern "C" cb_status cb_update(cb_ctx* ctx, const int32_t* tokens, int64_t row_s
                                const int32_t* n_new, void* stream) {
     CB_CHECK_ARG(ctx && tokens && n_old && n_new && row_stride >= 1);
     const int B = ctx->cfg.batch, wpb = 4;
-    CB_CUDA(cb_launch_pdl(cb_update_kernel, dim3((B + wpb - 1) / wpb), dim3(wpb * 32), 0, (cudaStream_t)stream, ctx->tables, B, tokens, row_stride,
+    CB_CUDA(cb_launch_pdl(ctx->cfg.FC <= 32 ? cb_update_kernel<true> : cb_update_kernel<false>, dim3((B + wpb - 1) / wpb), dim3(wpb * 32), 0, (cudaStream_t)stream, ctx->tables, B, tokens, row_stride,
                           n_old, n_new, ctx->d_status, ctx->d_counters));
     cb_count_launch(1);
     return CB_OK;
@@ -570,14 +625,15 @@ extern "C" cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t r
         static size_t opted[64] = {0};                         // largest size opted into so far, per device
         const int d = ctx->device & 63;
         if (opted[d] < smem) {
-            CB_CUDA(cudaFuncSetAttribute(cb_draft_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            CB_CUDA(cudaFuncSetAttribute(cb_draft_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            CB_CUDA(cudaFuncSetAttribute(cb_draft_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
             opted[d] = smem;
         }
     }
     const int threads = 32 * max(1, min(8, NL));
     CbTables tf = {};
     if (ctx->has_frozen) tf = ctx->frozen;
-    CB_CUDA(cb_launch_pdl(cb_draft_kernel, dim3(c.batch), dim3(threads), smem, (cudaStream_t)stream, ctx->tables, tf, T, c.crt, c.max_depth, NL, KF,
+    CB_CUDA(cb_launch_pdl(FCmax <= 32 ? cb_draft_kernel<true> : cb_draft_kernel<false>, dim3(c.batch), dim3(threads), smem, (cudaStream_t)stream, ctx->tables, tf, T, c.crt, c.max_depth, NL, KF,
                           tokens, row_stride, seq_len, tree_tokens, tree_parent, tree_depth, tree_mask, n_nodes, ctx->d_status, ctx->d_counters));
     cb_count_launch(1);
     return CB_OK;
