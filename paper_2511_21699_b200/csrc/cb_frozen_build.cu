@@ -11,7 +11,9 @@
 //   3. follower counts: windows whose leader was selected insert-or-increment the whole window in a second table; the
 //      distinct windows are then grouped by leader into one array (count per leader, exclusive scan, scatter);
 //   4. every distinct window scans its leader's group and counts the windows that beat it under (count falling, follower
-//      tokens rising), giving up at FC; a rank below FC is that follower's place in the entry.
+//      tokens rising), giving up at FC; a rank below FC is that follower's place in the entry.  A histogram of the counts'
+//      binary orders of magnitude per leader gives the order below which no window can be among the FC best, so that the
+//      many rare windows of a frequent leader leave at once.
 // Which occurrence represents a key, and which entry id a leader gets, depends on timing; the table's content (and
 // cb_frozen_dump's output) does not.
 #include "cb_common.cuh"
@@ -19,12 +21,14 @@
 namespace {
 
 constexpr uint32_t kEmpty = 0xFFFFFFFFu;
+constexpr uint32_t kBigGroup = 2048;          // distinct windows of one leader above which a window is ranked by a warp
 constexpr int kMaxWords = 1 + CB_MAX_LL;      // composite selection key: ~count, then the leader's tokens
 
 struct BuildState {                           // head of the scratch buffer
     uint32_t status;
     uint32_t n_uniq;                          // distinct leaders
     uint32_t n_sel;                           // entry ids handed out
+    uint32_t n_big;                           // windows of large groups that are ranked by a whole warp each
     uint32_t k_rem;                           // radix select: rank still to be resolved inside the current prefix
     uint32_t prefix[kMaxWords];               // composite key of the LC-th best leader, resolved digit by digit
     uint32_t select_all;                      // no more than LC distinct leaders: all of them are taken
@@ -38,6 +42,7 @@ struct BuildView {
     uint32_t* h2_pos; uint32_t* h2_cnt; int32_t* h2_eid;          // [S] windows of selected leaders
     uint32_t* seg; uint32_t* seg_cnt;                             // [S] distinct windows grouped by leader: slot, count
     uint32_t* grp_n; uint32_t* grp_off; uint32_t* grp_fill;       // [LC] group size, start, scatter cursor per entry
+    uint32_t* grp_hist;                                           // [LC][32] windows per floor(log2(count)); [0] becomes the cut-off order
     uint32_t S;                                                   // slots of each hash table (a power of two)
     const int32_t* corpus;
     uint32_t M;
@@ -88,6 +93,7 @@ __global__ void fb_init_kernel(BuildView v, CbTables t) {
         v.h2_pos[i] = kEmpty; v.h2_cnt[i] = 0u; v.h2_eid[i] = -1;
     }
     for (size_t i = g; i < (size_t)v.LC; i += stride) { v.grp_n[i] = 0u; v.grp_off[i] = 0u; v.grp_fill[i] = 0u; t.lstamp[i] = 0u; }
+    for (size_t i = g; i < (size_t)v.LC * 32; i += stride) v.grp_hist[i] = 0u;
     for (size_t i = g; i < t.nslots; i += stride) t.index[i] = CB_IDX_EMPTY;
     for (size_t i = g; i < (size_t)v.LC * t.E; i += stride) t.entries[i] = 0u;
     if (g < sizeof(BuildState) / 4) reinterpret_cast<uint32_t*>(v.st)[g] = 0u;
@@ -238,7 +244,23 @@ __global__ void fb_group_scatter_kernel(BuildView v) {
         const int32_t eid = v.h2_eid[s];
         const uint32_t at = v.grp_off[eid] + atomicAdd(&v.grp_fill[eid], 1u);
         v.seg[at] = (uint32_t)s;
-        v.seg_cnt[at] = v.h2_cnt[s];
+        const uint32_t c = v.h2_cnt[s];
+        v.seg_cnt[at] = c;
+        atomicAdd(&v.grp_hist[(size_t)eid * 32 + (31 - __clz(c))], 1u);
+    }
+}
+// 3d. per leader, the smallest order of magnitude that can still hold one of the FC most frequent windows
+__global__ void fb_group_cutoff_kernel(BuildView v) {
+    const uint32_t n = v.st->n_sel < (uint32_t)v.LC ? v.st->n_sel : (uint32_t)v.LC;
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (size_t)gridDim.x * blockDim.x) {
+        uint32_t* h = v.grp_hist + e * 32;
+        uint32_t acc = 0;
+        int b = 31;
+        for (; b > 0; --b) {
+            acc += h[b];
+            if (acc >= (uint32_t)v.FC) break;
+        }
+        h[0] = (uint32_t)b;                                  // orders below b hold none of the FC best
     }
 }
 
@@ -249,8 +271,13 @@ __global__ void fb_rank_followers_kernel(BuildView v, CbTables t) {
         if (v.h2_pos[s] == kEmpty) continue;
         const int32_t eid = v.h2_eid[s];
         const uint32_t mycnt = v.h2_cnt[s];
+        if ((uint32_t)(31 - __clz(mycnt)) < v.grp_hist[(size_t)eid * 32]) continue;   // FC windows of higher order exist
         const int32_t* mine = v.corpus + v.h2_pos[s] + v.LL;
         const uint32_t lo = v.grp_off[eid], hi = lo + v.grp_n[eid];
+        if (hi - lo > kBigGroup) {                           // a long scan: left to a warp (the list reuses the leaders' array)
+            v.uniq[atomicAdd(&v.st->n_big, 1u)] = (uint32_t)s;
+            continue;
+        }
         int rank = 0;
         for (uint32_t k = lo; k < hi && rank < v.FC; ++k) {
             const uint32_t c = v.seg_cnt[k];
@@ -272,11 +299,47 @@ __global__ void fb_rank_followers_kernel(BuildView v, CbTables t) {
     }
 }
 
+// 4b. the same for the windows of large groups, one warp per window: the lanes stride over the group
+__global__ void fb_rank_big_kernel(BuildView v, CbTables t) {
+    const int lane = threadIdx.x & 31;
+    const size_t nwarps = (size_t)gridDim.x * (blockDim.x >> 5);
+    const uint32_t n = v.st->n_big;
+    for (size_t w = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); w < n; w += nwarps) {
+        const uint32_t s = v.uniq[w];
+        const int32_t eid = v.h2_eid[s];
+        const uint32_t mycnt = v.h2_cnt[s];
+        const int32_t* mine = v.corpus + v.h2_pos[s] + v.LL;
+        const uint32_t lo = v.grp_off[eid], hi = lo + v.grp_n[eid];
+        int rank = 0;
+        for (uint32_t k0 = lo; k0 < hi && rank < v.FC; k0 += 32) {
+            const uint32_t k = k0 + lane;
+            bool beats = false;
+            if (k < hi) {
+                const uint32_t c = v.seg_cnt[k];
+                beats = c > mycnt;
+                if (c == mycnt) {
+                    const uint32_t o = v.seg[k];
+                    if (o != s) {
+                        const int32_t* other = v.corpus + v.h2_pos[o] + v.LL;
+                        for (int j = 0; j < v.FL; ++j)
+                            if (other[j] != mine[j]) { beats = other[j] < mine[j]; break; }
+                    }
+                }
+            }
+            rank += __popc(__ballot_sync(0xFFFFFFFFu, beats));
+        }
+        if (rank >= v.FC) continue;
+        uint32_t* e = t.entries + (size_t)eid * t.E;
+        if (lane < v.FL) e[v.LL + v.FC + rank * v.FL + lane] = (uint32_t)mine[lane];
+        if (lane == 0) e[v.LL + rank] = (uint32_t)(v.FC - rank);
+    }
+}
+
 size_t fb_align(size_t x) { return (x + 255) / 256 * 256; }
 
 struct BuildLayout {
     uint32_t S;
-    size_t off_h1_pos, off_h1_cnt, off_h1_eid, off_uniq, off_h2_pos, off_h2_cnt, off_h2_eid, off_seg, off_seg_cnt, off_grp, total;
+    size_t off_h1_pos, off_h1_cnt, off_h1_eid, off_uniq, off_h2_pos, off_h2_cnt, off_h2_eid, off_seg, off_seg_cnt, off_grp, off_hist, total;
 };
 
 cb_status fb_layout(const cb_frozen_config* c, int64_t n_tokens, BuildLayout* B) {
@@ -296,6 +359,7 @@ cb_status fb_layout(const cb_frozen_config* c, int64_t n_tokens, BuildLayout* B)
     B->off_seg = o;     o = fb_align(o + S * 4);
     B->off_seg_cnt = o; o = fb_align(o + S * 4);
     B->off_grp = o;     o = fb_align(o + (size_t)c->LC * 4 * 3);
+    B->off_hist = o;    o = fb_align(o + (size_t)c->LC * 4 * 32);
     B->total = o;
     return CB_OK;
 }
@@ -335,6 +399,7 @@ extern "C" cb_status cb_frozen_build(const cb_frozen_config* cfg, const int32_t*
     v.h2_pos = (uint32_t*)(base + B.off_h2_pos); v.h2_cnt = (uint32_t*)(base + B.off_h2_cnt); v.h2_eid = (int32_t*)(base + B.off_h2_eid);
     v.seg = (uint32_t*)(base + B.off_seg); v.seg_cnt = (uint32_t*)(base + B.off_seg_cnt);
     v.grp_n = (uint32_t*)(base + B.off_grp); v.grp_off = v.grp_n + cfg->LC; v.grp_fill = v.grp_off + cfg->LC;
+    v.grp_hist = (uint32_t*)(base + B.off_hist);
     v.S = B.S;
     v.corpus = dev_corpus;
     const int64_t M = n_tokens - cfg->LL - cfg->FL + 1;
@@ -357,8 +422,10 @@ extern "C" cb_status cb_frozen_build(const cb_frozen_config* cfg, const int32_t*
         fb_count_followers_kernel<<<grid, block, 0, st>>>(v);
         fb_group_scan_kernel<<<1, 1024, 0, st>>>(v);
         fb_group_scatter_kernel<<<grid, block, 0, st>>>(v);
+        fb_group_cutoff_kernel<<<grid, block, 0, st>>>(v);
         fb_rank_followers_kernel<<<grid, block, 0, st>>>(v, t);
-        cb_count_launch(7 + 8 * (1 + cfg->LL));
+        fb_rank_big_kernel<<<grid, block, 0, st>>>(v, t);
+        cb_count_launch(9 + 8 * (1 + cfg->LL));
     }
     cb_count_launch(1);
     CB_CUDA(cudaGetLastError());
