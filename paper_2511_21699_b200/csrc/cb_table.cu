@@ -381,6 +381,7 @@ struct DraftSmem {
     int32_t* tok; int32_t* par; int32_t* dep;
     int32_t* front; int32_t* next; int32_t* pts;
     int32_t* r_eid; int32_t* r_nf; int32_t* r_ok; uint32_t* r_stamp;
+    int32_t* r_n0; int32_t* r_cl; int32_t* r_tot; int32_t* r_nn0;     // plan of a leaf's attachment: first node, chain length, nodes, first frontier place
     int32_t* fol;
 };
 
@@ -398,7 +399,8 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
     S.tok = smem; S.par = S.tok + T; S.dep = S.par + T;
     S.front = S.dep + T; S.next = S.front + NL; S.pts = S.next + NL;
     S.r_eid = S.pts + NL; S.r_nf = S.r_eid + NL; S.r_ok = S.r_nf + NL; S.r_stamp = (uint32_t*)(S.r_ok + NL);
-    S.fol = (int32_t*)(S.r_stamp + NL);
+    S.r_n0 = (int32_t*)(S.r_stamp + NL); S.r_cl = S.r_n0 + NL; S.r_tot = S.r_cl + NL; S.r_nn0 = S.r_tot + NL;
+    S.fol = S.r_nn0 + NL;
     __shared__ int sh_n, sh_nfront, sh_nnext, sh_npts, sh_q, sh_hits, sh_fq, sh_fhits;
 
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -486,14 +488,34 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
                             int rank[CB_MAX_FC / 32];
 #pragma unroll
                             for (int c = 0; c < CB_MAX_FC / 32; ++c) rank[c] = -1;
-                            for (int r = 0; r < nf; ++r) {
-                                uint32_t m = fs[0];
+                            if (nf <= 16) {
+                                for (int r = 0; r < nf; ++r) {
+                                    uint32_t m = fs[0];
 #pragma unroll
-                                for (int c = 1; c < CB_MAX_FC / 32; ++c) m = max(m, fs[c]);
-                                const uint32_t g = __reduce_max_sync(CB_FULL, m);
+                                    for (int c = 1; c < CB_MAX_FC / 32; ++c) m = max(m, fs[c]);
+                                    const uint32_t g = __reduce_max_sync(CB_FULL, m);
+#pragma unroll
+                                    for (int c = 0; c < CB_MAX_FC / 32; ++c)
+                                        if (fs[c] == g) { rank[c] = r; fs[c] = 0u; }
+                                }
+                            } else {
+                                // many are wanted: rank every follower by counting the larger stamps (independent shuffles,
+                                // where the repeated maximum is a chain of reductions)
+                                int cntr[CB_MAX_FC / 32];
+#pragma unroll
+                                for (int c = 0; c < CB_MAX_FC / 32; ++c) cntr[c] = 0;
+#pragma unroll
+                                for (int c2 = 0; c2 < CB_MAX_FC / 32; ++c2) {
+                                    if (c2 * 32 >= tt.FC) break;
+                                    for (int l = 0; l < 32; ++l) {
+                                        const uint32_t o = __shfl_sync(CB_FULL, fs[c2], l);
+#pragma unroll
+                                        for (int c = 0; c < CB_MAX_FC / 32; ++c) cntr[c] += (o > fs[c]) ? 1 : 0;
+                                    }
+                                }
 #pragma unroll
                                 for (int c = 0; c < CB_MAX_FC / 32; ++c)
-                                    if (fs[c] == g) { rank[c] = r; fs[c] = 0u; }
+                                    if (fs[c] != 0u && cntr[c] < nf) rank[c] = cntr[c];
                             }
                             // every lane copies the tokens of its picked followers
 #pragma unroll
@@ -515,13 +537,17 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
                     if (lane == 0) { S.r_eid[li] = eid; S.r_nf[li] = nf; S.r_ok[li] = ok ? 1 : 0; }
                 }
                 __syncthreads();
-                // (2) sequential replay of the breadth-first order.  A query at the root (the only leaf of level 1) is issued,
-                // and its followers attached, while the tree has fewer than max(1, T - crt) nodes; any other while fewer than T.
+                // (2) the sequential breadth-first order, planned by one thread and filled in by all.  A query at the root (the only
+                // leaf of level 1) is issued, and its followers attached, while the tree has fewer than max(1, T - crt) nodes; any
+                // other while fewer than T.  Below a leaf of depth d every follower is a chain of min(FL, max_depth - d) nodes, the
+                // chains follow one another until the cap cuts the last one short, and a chain of FL nodes ends in a leaf of the
+                // next level: so a leaf's nodes and frontier places follow from where it starts, and only that is sequential.
+                const int lend = min(nfront, base + BS);
                 if (tid == 0) {
                     int n = n_now, q = 0, hits = 0, nn = sh_nnext;
-                    const int lend = min(nfront, base + BS);
                     for (int l2 = base; l2 < lend; ++l2) {
-                        if (n >= T) break;
+                        S.r_tot[l2] = 0;
+                        if (n >= T) continue;
                         const int leaf = S.front[l2];
                         const int cap = leaf == 0 ? max(1, T - crt) : T;
                         if (n >= cap) continue;
@@ -530,21 +556,29 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
                         if (S.r_eid[l2] < 0) continue;
                         ++hits;
                         if (pass == 0) S.r_stamp[l2] = clock0 + (uint32_t)(sh_q + q);
-                        for (int f = 0; f < S.r_nf[l2]; ++f) {
-                            if (n >= cap) break;
-                            int p = leaf, k = 0;
-                            for (int j = 0; j < t.FL; ++j) {
-                                if (n >= cap || S.dep[p] >= max_depth) break;
-                                S.tok[n] = S.fol[l2 * FLFC + f * t.FL + j];
-                                S.par[n] = p; S.dep[n] = S.dep[p] + 1; p = n; ++n; ++k;
-                            }
-                            if (k == t.FL) S.next[nn++] = p;
-                        }
+                        const int cl = min(t.FL, max_depth - S.dep[leaf]);
+                        const int tot = min(max(S.r_nf[l2], 0) * cl, cap - n);
+                        S.r_n0[l2] = n; S.r_cl[l2] = cl; S.r_tot[l2] = tot; S.r_nn0[l2] = nn;
+                        n += tot;
+                        if (cl == t.FL) nn += tot / t.FL;
                     }
                     sh_n = n; sh_nnext = nn;
                     if (pass == 0) { sh_q += q; sh_hits += hits; } else { sh_fq += q; sh_fhits += hits; }
                 }
                 __syncthreads();
+                for (int l2 = base; l2 < lend; ++l2) {
+                    const int tot = S.r_tot[l2];
+                    if (tot == 0) continue;
+                    const int leaf = S.front[l2], n0 = S.r_n0[l2], cl = S.r_cl[l2], d = S.dep[leaf];
+                    for (int x = tid; x < tot; x += blockDim.x) {
+                        const int f = x / cl, j = x - f * cl;
+                        S.tok[n0 + x] = S.fol[l2 * FLFC + f * t.FL + j];
+                        S.par[n0 + x] = j == 0 ? leaf : n0 + x - 1;
+                        S.dep[n0 + x] = d + j + 1;
+                    }
+                    if (cl == t.FL)
+                        for (int c = tid; c < tot / t.FL; c += blockDim.x) S.next[S.r_nn0[l2] + c] = n0 + c * t.FL + t.FL - 1;
+                }
             }
             // (3) stamp the leaders the sequential order reached; publish the next frontier
             if (pass == 0)
@@ -619,7 +653,7 @@ extern "C" cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t r
     // A leaf can receive at most T - 1 followers (each adds a node), so no more than that many are staged per lookup.
     const int FCmax = ctx->has_frozen ? max(c.FC, ctx->frozen.FC) : c.FC;
     const int KF = max(1, min(FCmax, T - 1));
-    const size_t smem = sizeof(int32_t) * ((size_t)3 * T + (size_t)7 * NL + (size_t)NL * c.FL * KF);
+    const size_t smem = sizeof(int32_t) * ((size_t)3 * T + (size_t)11 * NL + (size_t)NL * c.FL * KF);
     if (smem > 200 * 1024) return CB_ERR_UNSUPPORTED;
     if (smem > 48 * 1024) {
         static size_t opted[64] = {0};                         // largest size opted into so far, per device
