@@ -20,11 +20,14 @@ struct Probe {
 // through to L2 instead of from an L1 line that may be stale.
 // FETCH (tables with FC <= 32, so that lane l owns follower l alone): the follower's stamp and tokens are loaded together
 // with the key when an index word's tag matches, which saves the callers two dependent memory round trips.
+// FETCH == 2 (larger FC): the stamps of all the lane's followers come with the key (one round trip saved); the tokens are
+// loaded when they are known to be needed.
 struct EntryRegs {
     uint32_t fs;
     int32_t tok[CB_MAX_FL];
+    uint32_t fs4[CB_MAX_FC / 32];
 };
-template <bool SHARED = false, bool FETCH = false>
+template <bool SHARED = false, int FETCH = 0>
 __device__ __forceinline__ Probe tbl_find(const CbTables& t, const CbSeq& s, int32_t mykey, uint64_t h, int lane, EntryRegs* er = nullptr) {
     Probe r;
     r.eid = -2; r.slot = 0; r.free_slot = 0xFFFFFFFFu; r.probes = 0;
@@ -39,7 +42,13 @@ __device__ __forceinline__ Probe tbl_find(const CbTables& t, const CbSeq& s, int
             cand &= cand - 1;
             const uint32_t eid = __shfl_sync(CB_FULL, w, l) & CB_EID_MASK;
             bool eq = true;
-            if (FETCH) {
+            if (FETCH == 2) {
+                const uint32_t* e = s.entries + (size_t)eid * t.E;
+                const uint32_t kv = lane < t.LL ? e[lane] : 0u;
+#pragma unroll
+                for (int c = 0; c < CB_MAX_FC / 32; ++c) er->fs4[c] = (c * 32 + lane) < t.FC ? e[t.LL + c * 32 + lane] : 0u;
+                if (lane < t.LL) eq = (int32_t)kv == mykey;
+            } else if (FETCH == 1) {
                 const uint32_t* e = s.entries + (size_t)eid * t.E;
                 const bool mine = lane < t.FC;
                 const uint32_t kv = lane < t.LL ? e[lane] : 0u;
@@ -134,15 +143,20 @@ __device__ __forceinline__ void tbl_put_follower_regs(const CbTables& t, uint32_
     if (lane == 0) e[t.LL + tgt] = c;
 }
 
-__device__ __forceinline__ void tbl_put_follower(const CbTables& t, uint32_t* e, int32_t myfol, uint32_t c, int lane, TblCounters& cnt) {
+template <bool PRE = false>
+__device__ __forceinline__ void tbl_put_follower(const CbTables& t, uint32_t* e, int32_t myfol, uint32_t c, int lane, TblCounters& cnt,
+                                                 const EntryRegs* er = nullptr) {
     // Lane l looks after followers l, l + 32, ...: one pass finds a stored copy of the follower, the lowest free place
-    // and the least recently inserted follower.
+    // and the least recently inserted follower.  PRE: the stamps came with the lookup.
     int match_f = -1, free_f = -1, lru_f = -1;
     uint32_t lru_stamp = 0xFFFFFFFFu;
-    for (int base = 0; base < t.FC && match_f < 0; base += 32) {
+#pragma unroll
+    for (int ch = 0; ch < CB_MAX_FC / 32; ++ch) {
+        const int base = ch * 32;
+        if (base >= t.FC || match_f >= 0) break;
         const int f = base + lane;
         const bool mine = f < t.FC;
-        const uint32_t fs = mine ? e[t.LL + f] : 0u;
+        const uint32_t fs = PRE ? er->fs4[ch] : (mine ? e[t.LL + f] : 0u);
         bool match = mine && fs != 0u;
         for (int j = 0; j < t.FL; ++j) {
             const int32_t fj = __shfl_sync(CB_FULL, myfol, j);
@@ -166,7 +180,7 @@ __device__ __forceinline__ void tbl_put_follower(const CbTables& t, uint32_t* e,
 }
 
 // One insertion (Section 3.1). mykey = leader[lane] (lane < LL), myfol = follower[lane] (lane < FL).
-template <bool FETCH = false>
+template <int FETCH = 0>
 __device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int32_t myfol, uint32_t& clock,
                            uint32_t& count, int lane, uint32_t* status, TblCounters& cnt) {
     const uint32_t c = ++clock;
@@ -178,7 +192,8 @@ __device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int
     if (pr.eid >= 0) {
         uint32_t* e = s.entries + (size_t)pr.eid * t.E;
         if (lane == 0) s.lstamp[pr.eid] = c;
-        if (FETCH) tbl_put_follower_regs(t, e, er, myfol, c, lane, cnt);
+        if (FETCH == 1) tbl_put_follower_regs(t, e, er, myfol, c, lane, cnt);
+        else if (FETCH == 2) tbl_put_follower<true>(t, e, myfol, c, lane, cnt, &er);
         else tbl_put_follower(t, e, myfol, c, lane, cnt);
     } else if (pr.eid == -1) {
         int eid;
@@ -208,7 +223,7 @@ __device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int
 }
 
 // One warp per sequence; windows are applied in increasing position.
-template <bool FETCH>
+template <int FETCH>
 __global__ void __launch_bounds__(128) cb_update_kernel(CbTables t, int B, const int32_t* __restrict__ tokens,
                                                         int64_t row_stride, const int32_t* __restrict__ n_old,
                                                         const int32_t* __restrict__ n_new, uint32_t* status,
@@ -385,7 +400,7 @@ struct DraftSmem {
     int32_t* fol;
 };
 
-template <bool FETCH>
+template <int FETCH>
 __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, int T, int crt, int max_depth, int NL, int KF,
                                                        const int32_t* __restrict__ tokens, int64_t row_stride,
                                                        const int32_t* __restrict__ seq_len,
@@ -480,7 +495,8 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
                             uint32_t fs[CB_MAX_FC / 32];
 #pragma unroll
                             for (int c = 0; c < CB_MAX_FC / 32; ++c) {
-                                if (FETCH) fs[c] = c == 0 ? er.fs : 0u;            // FC <= 32: stamp and tokens came with the lookup
+                                if (FETCH == 1) fs[c] = c == 0 ? er.fs : 0u;       // FC <= 32: stamp and tokens came with the lookup
+                                else if (FETCH == 2) fs[c] = er.fs4[c];            // the stamps came with the lookup
                                 else fs[c] = (c * 32 + lane) < tt.FC ? e[tt.LL + c * 32 + lane] : 0u;
                                 nf += __popc(__ballot_sync(CB_FULL, fs[c] != 0u));
                             }
@@ -522,7 +538,7 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
                             for (int c = 0; c < CB_MAX_FC / 32; ++c) {
                                 if (rank[c] >= 0) {
                                     const int f = c * 32 + lane;
-                                    if (FETCH) {
+                                    if (FETCH == 1) {
 #pragma unroll
                                         for (int j = 0; j < CB_MAX_FL; ++j)
                                             if (j < tt.FL) S.fol[li * FLFC + rank[c] * tt.FL + j] = er.tok[j];
@@ -620,7 +636,7 @@ extern "C" cb_status cb_update(cb_ctx* ctx, const int32_t* tokens, int64_t row_s
                                const int32_t* n_new, void* stream) {
     CB_CHECK_ARG(ctx && tokens && n_old && n_new && row_stride >= 1);
     const int B = ctx->cfg.batch, wpb = 4;
-    CB_CUDA(cb_launch_pdl(ctx->cfg.FC <= 32 ? cb_update_kernel<true> : cb_update_kernel<false>, dim3((B + wpb - 1) / wpb), dim3(wpb * 32), 0, (cudaStream_t)stream, ctx->tables, B, tokens, row_stride,
+    CB_CUDA(cb_launch_pdl(ctx->cfg.FC <= 32 ? cb_update_kernel<1> : cb_update_kernel<2>, dim3((B + wpb - 1) / wpb), dim3(wpb * 32), 0, (cudaStream_t)stream, ctx->tables, B, tokens, row_stride,
                           n_old, n_new, ctx->d_status, ctx->d_counters));
     cb_count_launch(1);
     return CB_OK;
@@ -659,15 +675,15 @@ extern "C" cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t r
         static size_t opted[64] = {0};                         // largest size opted into so far, per device
         const int d = ctx->device & 63;
         if (opted[d] < smem) {
-            CB_CUDA(cudaFuncSetAttribute(cb_draft_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            CB_CUDA(cudaFuncSetAttribute(cb_draft_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            CB_CUDA(cudaFuncSetAttribute(cb_draft_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            CB_CUDA(cudaFuncSetAttribute(cb_draft_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
             opted[d] = smem;
         }
     }
     const int threads = 32 * max(1, min(8, NL));
     CbTables tf = {};
     if (ctx->has_frozen) tf = ctx->frozen;
-    CB_CUDA(cb_launch_pdl(FCmax <= 32 ? cb_draft_kernel<true> : cb_draft_kernel<false>, dim3(c.batch), dim3(threads), smem, (cudaStream_t)stream, ctx->tables, tf, T, c.crt, c.max_depth, NL, KF,
+    CB_CUDA(cb_launch_pdl(FCmax <= 32 ? cb_draft_kernel<1> : cb_draft_kernel<2>, dim3(c.batch), dim3(threads), smem, (cudaStream_t)stream, ctx->tables, tf, T, c.crt, c.max_depth, NL, KF,
                           tokens, row_stride, seq_len, tree_tokens, tree_parent, tree_depth, tree_mask, n_nodes, ctx->d_status, ctx->d_counters));
     cb_count_launch(1);
     return CB_OK;
