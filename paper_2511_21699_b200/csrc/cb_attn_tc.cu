@@ -46,6 +46,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t n) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(n) : "memory");
+}
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
@@ -306,7 +309,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             for (int s = 0; s < C::NSLOT; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_free(s), 1); }
             mbar_init(bar_qfull, 1); mbar_init(bar_qfree, 1); mbar_init(bar_sfull0, 1);
             for (int s = 0; s < 2; ++s) {
-                mbar_init(bar_pready(s), 128); mbar_init(bar_ofree(s), 128);
+                mbar_init(bar_pready(s), 256); mbar_init(bar_ofree(s), 128);
             }
             mbar_init(bar_cready, p.cs > 0 ? (uint32_t)p.cs : 1u); mbar_init(bar_cdata, 128);
             *s_abort = 0;
@@ -556,10 +559,13 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             if (wg == 1 && !two) {
                 // Handled by warpgroup 0 alone.  This warpgroup still watches every S completion, in order: waiting on a
                 // barrier by parity is only sound for a thread that is at most one phase away from it, and a thread that
-                // ran ahead over this unit would later meet ring barriers that are whole revolutions behind it.
+                // ran ahead over this unit would later meet ring barriers that are whole revolutions behind it.  It must
+                // not fall behind either (it may start late, after a long epilogue): half of every "P ready" arrival is
+                // its own, given when it has seen the tile's S, so the products cannot run more than a tile ahead of it.
                 for (int i = u.t0; ok && i < u.t1; ++i) {
                     const uint32_t kseq = seq0 + 2u * (uint32_t)(i - u.t0);
                     ok = mbar_wait(bar_free(kseq % C::NSLOT), (kseq / C::NSLOT) & 1, s_abort, p.status);
+                    mbar_arrive(bar_pready((i - u.t0) & 1));
                 }
                 have = fetch_next();
                 continue;
@@ -679,7 +685,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     tmem_wait_st();
                 }
                 tc_fence_before();
-                mbar_arrive(bar_pready(buf));
+                mbar_arrive_n(bar_pready(buf), two ? 2u : 1u);   // 256 arrivals per phase: the other half is the watching warpgroup's
             }
             if (!ok) break;
             have = fetch_next();

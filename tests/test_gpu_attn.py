@@ -123,3 +123,35 @@ def test_attn_full_size_sampled(oracle, name, full):
 
 def test_attn_config5_sampled(oracle):
     _run(W.get_config("c5_70b_long"), oracle, True, _sampled(1, 2, 4))
+
+
+def test_attn_long_units_mixed_row_tiles_repeated(oracle):
+    """Long contexts (257 key tiles per unit) with trees of one and of two row tiles side by side, launched several times: the
+    warpgroup that only watches a one-row-tile unit starts late after a two-row-tile epilogue and must neither run ahead of
+    the products nor fall behind them."""
+    from dataclasses import replace
+    from paper_2511_21699_b200 import Cacheback
+    cfg = replace(W.get_config("c5_70b_long"), name="c5_mixed", batch=24)
+    prob = Problem(cfg)
+    B, T = cfg.batch, cfg.max_nodes
+    par, dep, mask, n = synthetic_trees(cfg, full=False)
+    n[::3] = np.minimum(n[::3], 12)                       # every third tree fits one row tile (16 nodes with 8 heads per group)
+    for b in range(0, B, 3):
+        par[b], dep[b] = W.random_tree(cfg.seed, b, int(n[b]), cfg.max_depth, T)
+        mask[b] = W.tree_mask_from_parents(par[b], int(n[b]), (T + 31) // 32)
+    d = device_attn_inputs(cfg, prob)
+    cb = Cacheback.from_config(cfg)
+    lse = torch.zeros((B, cfg.n_q_heads, T), dtype=torch.float32, device="cuda")
+    out = torch.empty((B, T, cfg.n_q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda")
+    mask_d, n_d = dev(mask.view(np.int32)), dev(n)
+    for rep in range(6):
+        cb.cb_tree_attn(d["q"], d["k_pool"], d["v_pool"], d["block_table"], d["ctx_len"], d["k_tree"], d["v_tree"], mask_d, n_d,
+                        out=out, lse=lse, max_ctx=int(prob.ctx.max()))
+        torch.cuda.synchronize()
+        assert cb.cb_poll_status()[0] == 0, rep
+    for b in (0, 1, 3, 23):
+        rows = [(h, i) for h in (0, 37, 63) for i in sorted({0, int(n[b]) - 1, int(n[b]) // 2})]
+        ref, ref_lse = oracle_attn_rows(oracle, cfg, prob, mask, b, rows)
+        hh = torch.tensor([r[0] for r in rows], device="cuda")
+        ii = torch.tensor([r[1] for r in rows], device="cuda")
+        _check_rows(bf16_to_f64(out[b, ii, hh]), lse[b, hh, ii].cpu().numpy().astype(np.float64), ref, ref_lse, (cfg.name, b))
