@@ -43,8 +43,8 @@ def parse():
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one cb_attn_tc_kernel launch, from the ncu capture
 # summarised in profiles/cb_attn_tc_kernel_<workload>.md.  It is reported only while the kernel sources still hash to the
 # captured ones; after any change to them the figure is stale and `traffic` is null until the capture is redone.
-ATTN_TRAFFIC = {"sources_sha1": "de9264ffa8b7e161fd1ecad7147eb12c4cd1cad0",
-                "bytes_per_launch": {"c2_7b": 70.64e6, "c3_8b_gqa": 590.7e6, "c4_13b_turns": 2789.8e6}}
+ATTN_TRAFFIC = {"sources_sha1": "20295a8a7f97fe36322e3883899d465bc400bdc1",
+                "bytes_per_launch": {"c2_7b": 70.62e6, "c3_8b_gqa": 591.1e6, "c4_13b_turns": 2788.9e6}}
 
 
 def attn_sources_sha1():
