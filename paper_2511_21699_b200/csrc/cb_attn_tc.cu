@@ -606,8 +606,61 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     }
                     // rows that do not exist take the fast path too: whatever they compute stays in their own row
                     const bool all_vis = __all_sync(CB_FULL, !row_valid || (vm[0] & vm[1] & vm[2] & vm[3]) == 0xFFFFFFFFu);
-                    // pass 1: row maximum of the visible scores, 32 columns at a time with the next 32 in flight
                     uint32_t sa[32], sb[32];
+                    // Single pass, tried first on every tile but a share's first: P against the reference maximum in use,
+                    // the tile's own maximum alongside.  P is held back in registers, so S is still whole if a row turns out
+                    // to need a new reference (rare once a few tiles are in); then the two passes below run instead.  Both
+                    // ways give the same bits: the same operations on the same values in the same order.
+                    bool single = false;
+                    if (i > u.t0) {
+                        uint32_t pk[64];
+                        CB_TMEM_LD32(sa, 0, ts);
+                        const float mu = (m_used == -INFINITY) ? 0.f : m_used;
+                        const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), negmu2 = f2_pack(-mu, -mu);
+                        uint64_t lsa = f2_pack(0.f, 0.f), lsb = f2_pack(0.f, 0.f);
+                        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t* cur = (c & 1) ? sb : sa;
+                            uint32_t* nxt = (c & 1) ? sa : sb;
+                            CB_TMEM_WAIT_LD32(cur);
+                            if (c < 3) CB_TMEM_LD32(nxt, 0, ts + 32 * (c + 1));
+                            if (!all_vis) {
+#pragma unroll
+                                for (int jx = 0; jx < 32; ++jx)
+                                    if (!((vm[c] >> jx) & 1u)) cur[jx] = 0xFF800000u;
+                            }
+#pragma unroll
+                            for (int jx = 0; jx < 32; jx += 4) {
+                                const float s0 = __uint_as_float(cur[jx]), s1 = __uint_as_float(cur[jx + 1]);
+                                const float s2 = __uint_as_float(cur[jx + 2]), s3 = __uint_as_float(cur[jx + 3]);
+                                m0 = fmaxf(m0, s0); m1 = fmaxf(m1, s1); m2 = fmaxf(m2, s2); m3 = fmaxf(m3, s3);
+                                float p0, p1, p2, p3;
+                                f2_unpack(f2_fma(f2_pack(s0, s1), scale2, negmu2), p0, p1);
+                                f2_unpack(f2_fma(f2_pack(s2, s3), scale2, negmu2), p2, p3);
+                                p0 = ex2(p0); p1 = ex2(p1); p2 = ex2(p2); p3 = ex2(p3);
+                                lsa = f2_add(lsa, f2_pack(p0, p1));
+                                lsb = f2_add(lsb, f2_pack(p2, p3));
+                                pk[c * 16 + (jx >> 1)] = pack_bf16(p0, p1);
+                                pk[c * 16 + (jx >> 1) + 1] = pack_bf16(p2, p3);
+                            }
+                        }
+                        const float mloc = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * p.scale_log2;
+                        if (!__any_sync(CB_FULL, mloc > m_used + 8.0f)) {
+                            CB_TMEM_ST16(pk, 0, ts);
+                            CB_TMEM_ST16(pk, 16, ts + 16);
+                            CB_TMEM_ST16(pk, 32, ts + 32);
+                            CB_TMEM_ST16(pk, 48, ts + 48);
+                            float l0, l1, l2, l3;
+                            f2_unpack(lsa, l0, l1);
+                            f2_unpack(lsb, l2, l3);
+                            l += (l0 + l1) + (l2 + l3);
+                            tmem_wait_st();
+                            single = true;
+                        }
+                    }
+                    if (!single) {
+                    // pass 1: row maximum of the visible scores, 32 columns at a time with the next 32 in flight
                     CB_TMEM_LD32(sa, 0, ts);
                     float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
@@ -683,6 +736,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     f2_unpack(lsb, l2, l3);
                     l += (l0 + l1) + (l2 + l3);
                     tmem_wait_st();
+                    }
                 }
                 tc_fence_before();
                 mbar_arrive_n(bar_pready(buf), two ? 2u : 1u);   // 256 arrivals per phase: the other half is the watching warpgroup's
