@@ -33,6 +33,7 @@ namespace {
 
 constexpr long long kWaitCycles = 1ll << 32;     // bound of every wait, in SM clock cycles (about two seconds)
 constexpr uint32_t kSuspendNs = 20000;
+constexpr float kRowSumLimit = 1048576.f;        // a tile's row sum of P above which the row takes a new reference maximum
 constexpr int kThreads = 384;
 constexpr uint32_t kTmemCols = 512;
 
@@ -607,10 +608,12 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     // rows that do not exist take the fast path too: whatever they compute stays in their own row
                     const bool all_vis = __all_sync(CB_FULL, !row_valid || (vm[0] & vm[1] & vm[2] & vm[3]) == 0xFFFFFFFFu);
                     uint32_t sa[32], sb[32];
-                    // Single pass, tried first on every tile but a share's first: P against the reference maximum in use,
-                    // the tile's own maximum alongside.  P is held back in registers, so S is still whole if a row turns out
-                    // to need a new reference (rare once a few tiles are in); then the two passes below run instead.  Both
-                    // ways give the same bits: the same operations on the same values in the same order.
+                    // Single pass, tried first on every tile but a share's first: P against the reference maximum in use, held
+                    // back in registers so that S is still whole if the tile has to be done again.  No maximum is taken here.
+                    // The reference exists to keep 2^(s - reference) and its sums inside fp32 (P is bf16, same exponent
+                    // range), not for precision, so the tile's row sum tells all that matters: while it stays below
+                    // 2^20 no score is more than 20 above the reference and the tile stands; above that (or not finite)
+                    // the two passes below run instead and move the reference to the new maximum.
                     bool single = false;
                     if (i > u.t0) {
                         uint32_t pk[64];
@@ -618,7 +621,6 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                         const float mu = (m_used == -INFINITY) ? 0.f : m_used;
                         const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), negmu2 = f2_pack(-mu, -mu);
                         uint64_t lsa = f2_pack(0.f, 0.f), lsb = f2_pack(0.f, 0.f);
-                        float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             uint32_t* cur = (c & 1) ? sb : sa;
@@ -632,12 +634,9 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                             }
 #pragma unroll
                             for (int jx = 0; jx < 32; jx += 4) {
-                                const float s0 = __uint_as_float(cur[jx]), s1 = __uint_as_float(cur[jx + 1]);
-                                const float s2 = __uint_as_float(cur[jx + 2]), s3 = __uint_as_float(cur[jx + 3]);
-                                m0 = fmaxf(m0, s0); m1 = fmaxf(m1, s1); m2 = fmaxf(m2, s2); m3 = fmaxf(m3, s3);
                                 float p0, p1, p2, p3;
-                                f2_unpack(f2_fma(f2_pack(s0, s1), scale2, negmu2), p0, p1);
-                                f2_unpack(f2_fma(f2_pack(s2, s3), scale2, negmu2), p2, p3);
+                                f2_unpack(f2_fma(f2_pack(__uint_as_float(cur[jx]), __uint_as_float(cur[jx + 1])), scale2, negmu2), p0, p1);
+                                f2_unpack(f2_fma(f2_pack(__uint_as_float(cur[jx + 2]), __uint_as_float(cur[jx + 3])), scale2, negmu2), p2, p3);
                                 p0 = ex2(p0); p1 = ex2(p1); p2 = ex2(p2); p3 = ex2(p3);
                                 lsa = f2_add(lsa, f2_pack(p0, p1));
                                 lsb = f2_add(lsb, f2_pack(p2, p3));
@@ -645,16 +644,16 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                                 pk[c * 16 + (jx >> 1) + 1] = pack_bf16(p2, p3);
                             }
                         }
-                        const float mloc = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) * p.scale_log2;
-                        if (!__any_sync(CB_FULL, mloc > m_used + 8.0f)) {
+                        float l0, l1, l2, l3;
+                        f2_unpack(lsa, l0, l1);
+                        f2_unpack(lsb, l2, l3);
+                        const float lt = (l0 + l1) + (l2 + l3);
+                        if (!__any_sync(CB_FULL, !(lt <= kRowSumLimit))) {
                             CB_TMEM_ST16(pk, 0, ts);
                             CB_TMEM_ST16(pk, 16, ts + 16);
                             CB_TMEM_ST16(pk, 32, ts + 32);
                             CB_TMEM_ST16(pk, 48, ts + 48);
-                            float l0, l1, l2, l3;
-                            f2_unpack(lsa, l0, l1);
-                            f2_unpack(lsb, l2, l3);
-                            l += (l0 + l1) + (l2 + l3);
+                            l += lt;
                             tmem_wait_st();
                             single = true;
                         }
@@ -683,7 +682,8 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     float mloc = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
                     CB_TMEM_LD32(sa, 0, ts);                     // first columns of pass 2, in flight during the bookkeeping below
                     mloc *= p.scale_log2;
-                    // lazy rescaling: keep the reference maximum until the running maximum exceeds it by 2^8
+                    // lazy rescaling: keep the reference maximum until the running maximum exceeds it by 2^8 (a tile that
+                    // comes here from the single pass holds a score at least 2^13 above it)
                     const bool need = mloc > m_used + 8.0f;
                     const float alpha = need ? ex2(m_used - mloc) : 1.0f;
                     if (need) m_used = mloc;
