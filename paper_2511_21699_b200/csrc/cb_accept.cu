@@ -18,16 +18,22 @@ __device__ __forceinline__ unsigned long long pack(float x, uint32_t idx) {
 }
 __device__ __forceinline__ unsigned long long umax64(unsigned long long a, unsigned long long b) { return a > b ? a : b; }
 
-__device__ __forceinline__ float4 ldg_stream4(const float* p) {
+// The logits are read once: no L1 allocation, and first to leave L2 (the tables of the step's other kernels stay).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ float4 ldg_stream4(const float* p, uint64_t pol) {
     float4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.f32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(pol));
     return v;
 }
-__device__ __forceinline__ uint4 ldg_stream4u(const void* p) {
+__device__ __forceinline__ uint4 ldg_stream4u(const void* p, uint64_t pol) {
     uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
     return v;
 }
 
@@ -89,6 +95,7 @@ __global__ void __launch_bounds__(256) cb_accept_logits_kernel(
     if (i < n) {
         const int v0 = ck * chunk, v1 = min(V, v0 + chunk);
         unsigned long long best = 0ull;
+        const uint64_t pol = l2_evict_first_policy();
         if (!BF16) {
             const float* rowp = (const float*)logits + ((size_t)b * T + i) * row_stride;
             // head up to a 16-byte boundary, vector body, scalar tail
@@ -104,7 +111,7 @@ __global__ void __launch_bounds__(256) cb_accept_logits_kernel(
                 float4 x[4];
                 int kk[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) { kk[u] = k + u * blockDim.x; if (kk[u] < nvec) x[u] = ldg_stream4(base + 4 * (size_t)kk[u]); }
+                for (int u = 0; u < 4; ++u) { kk[u] = k + u * blockDim.x; if (kk[u] < nvec) x[u] = ldg_stream4(base + 4 * (size_t)kk[u], pol); }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) if (kk[u] < nvec) {
                     const uint32_t id = (uint32_t)(v + 4 * kk[u]);
@@ -130,7 +137,7 @@ __global__ void __launch_bounds__(256) cb_accept_logits_kernel(
                 uint4 x[4];
                 int kk[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) { kk[u] = k + u * blockDim.x; if (kk[u] < nvec) x[u] = ldg_stream4u(base + 8 * (size_t)kk[u]); }
+                for (int u = 0; u < 4; ++u) { kk[u] = k + u * blockDim.x; if (kk[u] < nvec) x[u] = ldg_stream4u(base + 8 * (size_t)kk[u], pol); }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) if (kk[u] < nvec) {
                     const uint32_t id = (uint32_t)(v + 8 * kk[u]);

@@ -120,6 +120,19 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 
+// The cached context is read once per call: its copies are marked as the first to leave L2, so that what the other kernels
+// of a step keep coming back to (the n-gram tables) is still there after 100 MB of keys and values have passed through.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3, uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cta.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -372,6 +385,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             const int within = lane % NB, j = within % 8, dblk = within / 8;
             uint32_t seq = 0;
             bool ok = true;
+            const uint64_t pol = l2_evict_first_policy();
             while (ok && wk.next(p, &u)) {
                 const int npages = (u.ctx + p.P - 1) / p.P, nct = u.tiles - 1;
                 const int32_t* bt = p.block_table + (size_t)u.b * p.max_pages;
@@ -389,7 +403,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     if (active) {
                         const uint32_t sl = isV ? vs : ks;
                         const uint32_t dst = sbase + C::OFF_RING + sl * C::TILE_BYTES + dblk * (CB_KT * 128) + j * 2048;
-                        if (i < nct) tma_load_4d(dst, isV ? &maps.v_pool : &maps.k_pool, bar_full(sl), dblk * 64, u.kh, 0, page);
+                        if (i < nct) tma_load_4d_hint(dst, isV ? &maps.v_pool : &maps.k_pool, bar_full(sl), dblk * 64, u.kh, 0, page, pol);
                         else tma_load_4d(dst, isV ? &maps.v_tree : &maps.k_tree, bar_full(sl), dblk * 64, u.kh, 16 * j, u.b);
                     }
                     seq += 2;
