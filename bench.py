@@ -2,7 +2,8 @@
 """Benchmark of the Cacheback draft-and-verify step on B200.
 
 A step is one pass of the whole hot path over one batch: cb_update (sliding window over the tokens
-accepted by the previous step) -> cb_draft_tree -> cb_tree_attn -> cb_accept (fp32 logits).  The default
+accepted by the previous step) -> cb_draft_tree -> cb_tree_attn -> cb_accept (fp32 logits); the first two are
+issued as the library's one-launch form cb_update_draft_tree unless --separate-calls is given.  The default
 workload is the Llama-2-7B-shaped configuration (batch 1, 32 heads, head_dim 128, context 4,096 in 16-token
 pages, tree cap 64).  Inputs are synthetic (seeded generators in workloads/).  Prints ONE JSON line.
 
@@ -35,6 +36,7 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--full-trees", action="store_true", help="attention/acceptance on synthetic full-size trees")
+    ap.add_argument("--separate-calls", action="store_true", help="cb_update and cb_draft_tree as two launches")
     ap.add_argument("--frozen", type=int, default=0, metavar="TOKENS",
                     help="attach a frozen table built on the GPU from a synthetic corpus of this many tokens (0 = none)")
     return ap.parse_args()
@@ -309,8 +311,11 @@ def run_ours(args, rank, world, local_rank):
     def step(s):
         r = s % R
         tr = trees[s]
-        cb.cb_update(toks_d, n_old[s], n_new[s])
-        cb.cb_draft_tree(toks_d, n_new[s], tr)
+        if args.separate_calls:
+            cb.cb_update(toks_d, n_old[s], n_new[s])
+            cb.cb_draft_tree(toks_d, n_new[s], tr)
+        else:
+            cb.cb_update_draft_tree(toks_d, n_old[s], n_new[s], tr)
         at = ftree if args.full_trees else tr
         cb.cb_tree_attn(q, kps[r], vps[r], bt_d, ctx_d, kt, vt, at["mask"], at["n_nodes"], out=out, max_ctx=int(ctx.max()))
         cb.cb_accept(at, logits=lgs[r], res=res)
@@ -365,14 +370,16 @@ def run_ours(args, rank, world, local_rank):
                 cb.cb_draft_tree(toks_d, n_new[s], tr)
             elif which == 2:
                 cb.cb_tree_attn(q, kps[r], vps[r], bt_d, ctx_d, kt, vt, at["mask"], at["n_nodes"], out=out, max_ctx=int(ctx.max()))
-            else:
+            elif which == 3:
                 cb.cb_accept(at, logits=lgs[r], res=res)
+            else:
+                cb.cb_update_draft_tree(toks_d, n_old[s], n_new[s], tr)
 
         for s in range(base, base + K):                      # one eager pass leaves valid trees for every step index
             step(s)
         stream.synchronize()
-        per_med = np.zeros(4)
-        for which in range(4):
+        per_med = np.zeros(5)
+        for which in range(5):
             gc = torch.cuda.CUDAGraph()
             with torch.cuda.graph(gc, stream=stream):
                 for s in range(base, base + K):
@@ -415,8 +422,11 @@ def run_ours(args, rank, world, local_rank):
             dlg.copy_(hlg, non_blocking=True)
             d_old.copy_(h_old[s], non_blocking=True); d_new.copy_(h_new[s], non_blocking=True)
             tr = trees[s]
-            cb.cb_update(toks_d, d_old, d_new)
-            cb.cb_draft_tree(toks_d, d_new, tr)
+            if args.separate_calls:
+                cb.cb_update(toks_d, d_old, d_new)
+                cb.cb_draft_tree(toks_d, d_new, tr)
+            else:
+                cb.cb_update_draft_tree(toks_d, d_old, d_new, tr)
             at = ftree if args.full_trees else tr
             cb.cb_tree_attn(dq, kps[r], vps[r], bt_d, ctx_d, dkt, dvt, at["mask"], at["n_nodes"], out=out, max_ctx=int(ctx.max()))
             cb.cb_accept(at, logits=dlg, res=res)
@@ -461,13 +471,14 @@ def run_ours(args, rank, world, local_rank):
                    "context": [int(ctx.min()), int(ctx.max())], "l2": "rotating %d copies of K/V pool and logits (%.0f MB)" %
                    (R, R * (pool_bytes + logit_bytes) / 1e6), "launch": "CUDA graph of the timed steps, replayed %d times, median" % reps,
                    "trees": "synthetic full" if args.full_trees else "drafted", "frozen_table": frozen_info,
+                   "calls": ("cb_update, cb_draft_tree" if args.separate_calls else "cb_update_draft_tree") + ", cb_tree_attn, cb_accept",
                    "parallelism": "replicas x%d" % world},
         "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "ms_per_step": 1e3 * e2e_s / K},
         "roofline": roof,
         "per_call_ms": {"cb_update": float(per_med[0]), "cb_draft_tree": float(per_med[1]), "cb_tree_attn": float(per_med[2]),
-                        "cb_accept": float(per_med[3])},
+                        "cb_accept": float(per_med[3]), "cb_update_draft_tree": float(per_med[4])},
         "accept_gbs": (float(np.sum(nn_mean)) * cfg.vocab * 4) / (float(per_med[3]) * 1e-3) / 1e9,
         "counters": counters,
     }

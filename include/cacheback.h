@@ -140,6 +140,16 @@ cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, 
                         uint32_t* tree_mask, int32_t* n_nodes, void* stream);
 
 /*
+ * cb_update followed by cb_draft_tree on the grown sequences, in one launch (Section 3.2: the table is brought up to
+ * date with the newly accepted tokens before the next draft is made from it).  Same arguments, results, table state
+ * and errors as cb_update(tokens, row_stride, n_old, n_new) followed by cb_draft_tree(tokens, row_stride, n_new, ...);
+ * at small batch the step saves a kernel boundary.
+ */
+cb_status cb_update_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* n_old,
+                               const int32_t* n_new, int32_t* tree_tokens, int32_t* tree_parent, int32_t* tree_depth,
+                               uint32_t* tree_mask, int32_t* n_nodes, void* stream);
+
+/*
  * Extra branches from another drafter (Conclusion: because the drafts form a tree, the predicted drafts of other
  * speculative-decoding methods can be inserted as additional branches).  Call it between cb_draft_tree and the
  * verification pass.

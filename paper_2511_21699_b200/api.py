@@ -185,6 +185,16 @@ class Cacheback:
                                       _ptr(tree["n_nodes"], torch.int32), _stream(stream)), "cb_draft_tree")
         return tree
 
+    def cb_update_draft_tree(self, tokens, n_old, n_new, tree=None, stream=None):
+        """cb_update(tokens, n_old, n_new) and cb_draft_tree(tokens, n_new) in one launch."""
+        tree = tree if tree is not None else self.alloc_tree()
+        _check(self.lib.cb_update_draft_tree(self._h, _ptr(tokens, torch.int32), tokens.stride(0), _ptr(n_old, torch.int32),
+                                             _ptr(n_new, torch.int32),
+                                             _ptr(tree["tokens"], torch.int32), _ptr(tree["parent"], torch.int32),
+                                             _ptr(tree["depth"], torch.int32), _ptr(tree["mask"], torch.int32),
+                                             _ptr(tree["n_nodes"], torch.int32), _stream(stream)), "cb_update_draft_tree")
+        return tree
+
     def cb_tree_add_branches(self, tree, branches, branch_len, stream=None):
         """branches int32 [batch, K, Lmax], branch_len int32 [batch, K]: extends `tree` in place."""
         K, Lmax = int(branches.shape[1]), int(branches.shape[2])

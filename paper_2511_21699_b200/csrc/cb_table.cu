@@ -224,17 +224,10 @@ __device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int
 
 // One warp per sequence; windows are applied in increasing position.
 template <int FETCH>
-__global__ void __launch_bounds__(128) cb_update_kernel(CbTables t, int B, const int32_t* __restrict__ tokens,
-                                                        int64_t row_stride, const int32_t* __restrict__ n_old,
-                                                        const int32_t* __restrict__ n_new, uint32_t* status,
-                                                        unsigned long long* counters) {
-    CB_PDL_ENTRY();
-    const int lane = threadIdx.x & 31;
-    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (b >= B) return;
+__device__ __forceinline__ void update_seq(const CbTables& t, int b, const int32_t* __restrict__ tokens, int64_t row_stride, int n0, int n1,
+                                           int lane, uint32_t* status, unsigned long long* counters) {
     const CbSeq s = cb_seq(t, b);
     const int w = t.LL + t.FL;
-    const int n0 = n_old[b], n1 = n_new[b];
     uint32_t clock = s.hdr[0], count = s.hdr[1];
     TblCounters cnt = {0, 0, 0, 0};
     const int32_t* row = tokens + (size_t)b * row_stride;
@@ -250,6 +243,18 @@ __global__ void __launch_bounds__(128) cb_update_kernel(CbTables t, int B, const
         if (cnt.fevict) atomicAdd(&counters[CB_CNT_FOLLOWER_EVICTIONS], (unsigned long long)cnt.fevict);
         if (cnt.maxprobe) atomicMax(&counters[CB_CNT_MAX_PROBE], (unsigned long long)cnt.maxprobe);
     }
+}
+
+template <int FETCH>
+__global__ void __launch_bounds__(128) cb_update_kernel(CbTables t, int B, const int32_t* __restrict__ tokens,
+                                                        int64_t row_stride, const int32_t* __restrict__ n_old,
+                                                        const int32_t* __restrict__ n_new, uint32_t* status,
+                                                        unsigned long long* counters) {
+    CB_PDL_ENTRY();
+    const int lane = threadIdx.x & 31;
+    const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (b >= B) return;
+    update_seq<FETCH>(t, b, tokens, row_stride, n_old[b], n_new[b], lane, status, counters);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -403,7 +408,7 @@ struct DraftSmem {
 template <int FETCH>
 __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, int T, int crt, int max_depth, int NL, int KF,
                                                        const int32_t* __restrict__ tokens, int64_t row_stride,
-                                                       const int32_t* __restrict__ seq_len,
+                                                       const int32_t* __restrict__ seq_len, const int32_t* __restrict__ upd_n_old,
                                                        int32_t* __restrict__ o_tok, int32_t* __restrict__ o_par,
                                                        int32_t* __restrict__ o_dep, uint32_t* __restrict__ o_mask,
                                                        int32_t* __restrict__ o_n, uint32_t* status,
@@ -422,6 +427,13 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
     const CbSeq s = cb_seq(t, b);
     const int32_t* row = tokens + (size_t)b * row_stride;
     const int L = seq_len[b];
+    if (upd_n_old != nullptr) {
+        // cb_update_draft_tree: the sequence's new windows go into the table first (one warp, in order, exactly as
+        // cb_update does), then the whole CTA drafts from the updated table.
+        if (warp == 0) update_seq<FETCH>(t, b, tokens, row_stride, upd_n_old[b], L, lane, status, counters);
+        __threadfence_block();
+        __syncthreads();
+    }
     const int W = (T + 31) >> 5;
     const int FLFC = t.FL * KF;                               // staged followers per leaf: the KF best
     const uint32_t clock0 = s.hdr[0];
@@ -658,9 +670,9 @@ extern "C" cb_status cb_update_bulk(cb_ctx* ctx, const int32_t* tokens, int64_t 
     return CB_OK;
 }
 
-extern "C" cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* seq_len,
-                                   int32_t* tree_tokens, int32_t* tree_parent, int32_t* tree_depth,
-                                   uint32_t* tree_mask, int32_t* n_nodes, void* stream) {
+static cb_status draft_launch(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* seq_len, const int32_t* upd_n_old,
+                              int32_t* tree_tokens, int32_t* tree_parent, int32_t* tree_depth,
+                              uint32_t* tree_mask, int32_t* n_nodes, void* stream) {
     CB_CHECK_ARG(ctx && tokens && seq_len && tree_tokens && tree_parent && tree_depth && tree_mask && n_nodes);
     CB_CHECK_ARG(row_stride >= 1);
     const cb_config& c = ctx->cfg;
@@ -684,7 +696,20 @@ extern "C" cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t r
     CbTables tf = {};
     if (ctx->has_frozen) tf = ctx->frozen;
     CB_CUDA(cb_launch_pdl(FCmax <= 32 ? cb_draft_kernel<1> : cb_draft_kernel<2>, dim3(c.batch), dim3(threads), smem, (cudaStream_t)stream, ctx->tables, tf, T, c.crt, c.max_depth, NL, KF,
-                          tokens, row_stride, seq_len, tree_tokens, tree_parent, tree_depth, tree_mask, n_nodes, ctx->d_status, ctx->d_counters));
+                          tokens, row_stride, seq_len, upd_n_old, tree_tokens, tree_parent, tree_depth, tree_mask, n_nodes, ctx->d_status, ctx->d_counters));
     cb_count_launch(1);
     return CB_OK;
+}
+
+extern "C" cb_status cb_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* seq_len,
+                                   int32_t* tree_tokens, int32_t* tree_parent, int32_t* tree_depth,
+                                   uint32_t* tree_mask, int32_t* n_nodes, void* stream) {
+    return draft_launch(ctx, tokens, row_stride, seq_len, nullptr, tree_tokens, tree_parent, tree_depth, tree_mask, n_nodes, stream);
+}
+
+extern "C" cb_status cb_update_draft_tree(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* n_old,
+                                          const int32_t* n_new, int32_t* tree_tokens, int32_t* tree_parent,
+                                          int32_t* tree_depth, uint32_t* tree_mask, int32_t* n_nodes, void* stream) {
+    CB_CHECK_ARG(n_old != nullptr);
+    return draft_launch(ctx, tokens, row_stride, n_new, n_old, tree_tokens, tree_parent, tree_depth, tree_mask, n_nodes, stream);
 }

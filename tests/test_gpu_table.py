@@ -114,6 +114,48 @@ def test_update_draft_accept_closed_loop(oracle, name, steps):
         assert total_accept > 0                  # the drafter does get tokens accepted on these streams
 
 
+@pytest.mark.parametrize("name,steps", [("c1_tiny", 16), ("c2_7b", 16), ("c3_8b_gqa", 6), ("c1_evict256", 16),
+                                        ("p_tuned", 10), ("p_fc40_evict", 10)])
+def test_update_draft_in_one_launch(oracle, name, steps):
+    """cb_update_draft_tree = cb_update then cb_draft_tree: same trees every step and the same table at the end as the
+    oracle's update followed by its draft."""
+    cfg = W.get_config(name)
+    prob = Problem(cfg)
+    B, T = cfg.batch, cfg.max_nodes
+    cb = _mk(cfg)
+    otabs = [oracle.OracleTable(cfg.LL, cfg.FL, cfg.LC, cfg.FC) for _ in range(B)]
+    toks_d = dev(prob.toks)
+    zero = torch.zeros(B, dtype=torch.int32, device="cuda")
+    pos = prob.prefill.copy()
+    if "evict" in name:
+        pos = (prob.lens - T - 2 - 8 * steps).astype(np.int32)
+    cb.cb_update(toks_d, zero, dev(pos))
+    for b in range(B):
+        otabs[b].update(prob.toks[b], 0, int(pos[b]))
+    prev = pos.copy()
+    tree = cb.alloc_tree()
+    for step in range(steps):
+        cb.cb_update_draft_tree(toks_d, dev(prev), dev(pos), tree)
+        g = {k: v.cpu().numpy() for k, v in tree.items()}
+        new_pos = pos.copy()
+        for b in range(B):
+            otabs[b].update(prob.toks[b], int(prev[b]), int(pos[b]))
+            n, tok, par, dep, mask = otabs[b].draft_tree(prob.toks[b], int(pos[b]), T, cfg.crt, cfg.max_depth)
+            assert g["n_nodes"][b] == n, (step, b)
+            assert np.array_equal(g["tokens"][b], tok) and np.array_equal(g["parent"][b], par), (step, b)
+            assert np.array_equal(g["depth"][b], dep), (step, b)
+            assert np.array_equal(g["mask"][b].view(np.uint32), mask), (step, b)
+            # the stream is the target: accept the matching path, plus the bonus token
+            m = oracle.accept(tok, par, dep, n, _stream_targets(prob.toks[b], int(pos[b]), n, tok, par, T, b, step), cfg.max_depth)[0]
+            new_pos[b] = min(pos[b] + m + 1 + (step % 3), prob.lens[b] - T - 2)
+        prev, pos = pos, new_pos
+    check = range(B) if B <= 8 else [0, 1, B // 2, B - 1]
+    _assert_tables_equal(cb, otabs, check)
+    st, cnt = cb.cb_poll_status()
+    assert st == 0, st
+    assert cnt["inserts"] > 0 and cnt["queries"] > 0
+
+
 @pytest.mark.parametrize("fixture", ["trace_a_lru.json", "trace_b_follower_refresh.json"])
 def test_hand_traces_on_gpu(fixture):
     g = golden(fixture)
