@@ -45,8 +45,8 @@ def parse():
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one cb_attn_tc_kernel launch, from the ncu capture
 # summarised in profiles/cb_attn_tc_kernel_<workload>.md.  It is reported only while the kernel sources still hash to the
 # captured ones; after any change to them the figure is stale and `traffic` is null until the capture is redone.
-ATTN_TRAFFIC = {"sources_sha1": "20295a8a7f97fe36322e3883899d465bc400bdc1",
-                "bytes_per_launch": {"c2_7b": 70.62e6, "c3_8b_gqa": 591.1e6, "c4_13b_turns": 2788.9e6}}
+ATTN_TRAFFIC = {"sources_sha1": "99d7999d0ae4e2f279e4d9d560031a8527d056dd",
+                "bytes_per_launch": {"c2_7b": 70.22e6, "c3_8b_gqa": 557.9e6, "c4_13b_turns": 2769.2e6}}
 
 
 def attn_sources_sha1():
