@@ -622,16 +622,33 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     // rows that do not exist take the fast path too: whatever they compute stays in their own row
                     const bool all_vis = __all_sync(CB_FULL, !row_valid || (vm[0] & vm[1] & vm[2] & vm[3]) == 0xFFFFFFFFu);
                     uint32_t sa[32], sb[32];
-                    // Single pass, tried first on every tile but a share's first: P against the reference maximum in use, held
-                    // back in registers so that S is still whole if the tile has to be done again.  No maximum is taken here.
-                    // The reference exists to keep 2^(s - reference) and its sums inside fp32 (P is bf16, same exponent
-                    // range), not for precision, so the tile's row sum tells all that matters: while it stays below
-                    // 2^20 no score is more than 20 above the reference and the tile stands; above that (or not finite)
-                    // the two passes below run instead and move the reference to the new maximum.
+                    // Single pass, tried first on every tile: P against the reference maximum in use, held back in registers so
+                    // that S is still whole if the tile has to be done again.  No row maximum is taken.  The reference exists
+                    // to keep 2^(s - reference) and its sums inside fp32 (P is bf16, same exponent range), not for precision,
+                    // so the tile's row sum tells all that matters: while it stays below 2^20 no score is more than 20
+                    // above the reference and the tile stands; above that (or not finite) the two passes below run instead
+                    // and move the reference to the new maximum.  A share's first tile has no reference yet and takes the
+                    // largest of its first 32 scores.
                     bool single = false;
-                    if (i > u.t0) {
+                    {
                         uint32_t pk[64];
                         CB_TMEM_LD32(sa, 0, ts);
+                        CB_TMEM_WAIT_LD32(sa);
+                        CB_TMEM_LD32(sb, 0, ts + 32);
+                        if (!all_vis) {
+#pragma unroll
+                            for (int jx = 0; jx < 32; ++jx)
+                                if (!((vm[0] >> jx) & 1u)) sa[jx] = 0xFF800000u;
+                        }
+                        if (i == u.t0) {
+                            float c0 = -INFINITY, c1 = -INFINITY, c2 = -INFINITY, c3 = -INFINITY;
+#pragma unroll
+                            for (int jx = 0; jx < 32; jx += 4) {
+                                c0 = fmaxf(c0, __uint_as_float(sa[jx])); c1 = fmaxf(c1, __uint_as_float(sa[jx + 1]));
+                                c2 = fmaxf(c2, __uint_as_float(sa[jx + 2])); c3 = fmaxf(c3, __uint_as_float(sa[jx + 3]));
+                            }
+                            m_used = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3)) * p.scale_log2;   // -inf if the row sees none of them
+                        }
                         const float mu = (m_used == -INFINITY) ? 0.f : m_used;
                         const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), negmu2 = f2_pack(-mu, -mu);
                         uint64_t lsa = f2_pack(0.f, 0.f), lsb = f2_pack(0.f, 0.f);
@@ -639,12 +656,14 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                         for (int c = 0; c < 4; ++c) {
                             uint32_t* cur = (c & 1) ? sb : sa;
                             uint32_t* nxt = (c & 1) ? sa : sb;
-                            CB_TMEM_WAIT_LD32(cur);
-                            if (c < 3) CB_TMEM_LD32(nxt, 0, ts + 32 * (c + 1));
-                            if (!all_vis) {
+                            if (c > 0) {
+                                CB_TMEM_WAIT_LD32(cur);
+                                if (c < 3) CB_TMEM_LD32(nxt, 0, ts + 32 * (c + 1));
+                                if (!all_vis) {
 #pragma unroll
-                                for (int jx = 0; jx < 32; ++jx)
-                                    if (!((vm[c] >> jx) & 1u)) cur[jx] = 0xFF800000u;
+                                    for (int jx = 0; jx < 32; ++jx)
+                                        if (!((vm[c] >> jx) & 1u)) cur[jx] = 0xFF800000u;
+                                }
                             }
 #pragma unroll
                             for (int jx = 0; jx < 32; jx += 4) {
