@@ -115,6 +115,53 @@ def test_attn_cluster_mode_empty_tree(oracle):
     assert cb.cb_poll_status()[0] == 0 and (out == 0).all()
 
 
+def _times16(bits):
+    """bf16 bit patterns times 16 (exact: four exponent steps)."""
+    f = (bits.astype(np.uint32) << 16).view(np.float32) * np.float32(16.0)
+    return (f.view(np.uint32) >> 16).astype(np.uint16)
+
+
+@pytest.mark.parametrize("cfg,ctxs", [(CLUSTER_4, [600]), (SMALL_GQA, [300, 300, 300, 257, 140])])
+def test_attn_score_jumps_between_and_inside_tiles(oracle, cfg, ctxs):
+    """Keys of the second key tile, and of the first tile past its first 40 keys, are 16 times larger: their scores lie
+    dozens of powers of two above the reference maximum the softmax has in use when it meets them (taken from an
+    earlier tile, or from the first 32 scores of a share's first tile), so the one-pass form must give way to the
+    form that takes the row maximum first.  Cluster mode and the stream-K split."""
+    from paper_2511_21699_b200 import Cacheback
+    prob = Problem(cfg)
+    prob.ctx = np.asarray(ctxs, np.int32)
+    prob.bt, prob.num_pages = W.make_block_table(cfg, prob.ctx)
+    B, T, P = cfg.batch, cfg.max_nodes, cfg.page_size
+    par, dep, mask, n = synthetic_trees(cfg, full=False)
+    kp, vp = W.pool_pages_bits(cfg, np.arange(prob.num_pages))
+    for b in range(B):
+        big = [t for t in range(int(prob.ctx[b])) if 128 <= t < 256 or (b == 0 and 40 <= t < 128)]
+        for t in big:
+            pg = prob.bt[b, t // P]
+            kp[pg, t % P] = _times16(kp[pg, t % P])
+    d = device_attn_inputs(cfg, prob)
+    d["k_pool"] = torch.from_numpy(kp.view(np.int16)).cuda().view(torch.bfloat16)
+    cb = Cacheback.from_config(cfg)
+    lse = torch.zeros((B, cfg.n_q_heads, T), dtype=torch.float32, device="cuda")
+    out = torch.empty((B, T, cfg.n_q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda")
+    cb.cb_tree_attn(d["q"], d["k_pool"], d["v_pool"], d["block_table"], d["ctx_len"], d["k_tree"], d["v_tree"],
+                    dev(mask.view(np.int32)), dev(n), out=out, lse=lse, max_ctx=int(prob.ctx.max()))
+    torch.cuda.synchronize()
+    assert cb.cb_poll_status()[0] == 0
+    for b in range(B):
+        npg = (int(prob.ctx[b]) + P - 1) // P
+        pages = prob.bt[b, :npg]
+        rows_hi = [(h, i) for h in sorted({0, 1, cfg.n_q_heads // 2, cfg.n_q_heads - 1}) for i in sorted({0, int(n[b]) // 2, int(n[b]) - 1})]
+        rows = np.array([(0, h, i) for h, i in rows_hi], dtype=np.int32)
+        ref, ref_lse = oracle.tree_attn_rows(W.seq_bits(cfg, W.tensors.TID.Q, b, cfg.n_q_heads)[None], kp[pages], vp[pages],
+                                             np.arange(npg, dtype=np.int32)[None], prob.ctx[b:b + 1],
+                                             W.seq_bits(cfg, W.tensors.TID.K_TREE, b, cfg.n_kv_heads)[None],
+                                             W.seq_bits(cfg, W.tensors.TID.V_TREE, b, cfg.n_kv_heads)[None], mask[b:b + 1], rows)
+        hh = torch.tensor([r[0] for r in rows_hi], device="cuda")
+        ii = torch.tensor([r[1] for r in rows_hi], device="cuda")
+        _check_rows(bf16_to_f64(out[b, ii, hh]), lse[b, hh, ii].cpu().numpy().astype(np.float64), ref, ref_lse, (cfg.name, b))
+
+
 @pytest.mark.parametrize("name", ["c2_7b", "c3_8b_gqa", "c4_13b_turns", "p_tuned"])
 @pytest.mark.parametrize("full", [True, False])
 def test_attn_full_size_sampled(oracle, name, full):
