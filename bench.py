@@ -45,8 +45,8 @@ def parse():
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one cb_attn_tc_kernel launch, from the ncu capture
 # summarised in profiles/cb_attn_tc_kernel_<workload>.md.  It is reported only while the kernel sources still hash to the
 # captured ones; after any change to them the figure is stale and `traffic` is null until the capture is redone.
-ATTN_TRAFFIC = {"sources_sha1": "99d7999d0ae4e2f279e4d9d560031a8527d056dd",
-                "bytes_per_launch": {"c2_7b": 70.22e6, "c3_8b_gqa": 557.9e6, "c4_13b_turns": 2769.2e6}}
+ATTN_TRAFFIC = {"sources_sha1": "940d4a8002e5bcb4876bd7445ef665e14f2a13aa",
+                "bytes_per_launch": {"c2_7b": 70.37e6, "c3_8b_gqa": 558.2e6, "c4_13b_turns": 2768.5e6}}
 
 
 def attn_sources_sha1():
