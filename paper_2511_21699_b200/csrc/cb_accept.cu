@@ -38,13 +38,11 @@ __device__ __forceinline__ uint4 ldg_stream4u(const void* p, uint64_t pol) {
 }
 
 // Walk of one sequence by one warp (n <= 128 nodes, parents precede children).
-__device__ void accept_walk(int b, int T, int Dmax, const int32_t* __restrict__ tok, const int32_t* __restrict__ par,
-                            const int32_t* __restrict__ dep, int n, const int32_t* target_s /*shared, [T]*/,
+// tk, pa, de: the sequence's own tree rows (shared or global memory).
+__device__ void accept_walk(int b, int Dmax, const int32_t* tk, const int32_t* pa, const int32_t* de, int n,
+                            const int32_t* target_s /*shared, [T]*/,
                             int32_t* __restrict__ n_accept, int32_t* __restrict__ accept_nodes,
                             int32_t* __restrict__ out_tokens, int lane) {
-    const int32_t* tk = tok + (size_t)b * T;
-    const int32_t* pa = par + (size_t)b * T;
-    const int32_t* de = dep + (size_t)b * T;
     // key = (depth << 8) | (255 - index) for verified nodes: max = deepest, lowest index among ties
     uint32_t best = 0;
     for (int i = lane; i < n; i += 32) {
@@ -90,7 +88,7 @@ __global__ void __launch_bounds__(256) cb_accept_logits_kernel(
     const int b = blockIdx.z, i = blockIdx.y, ck = blockIdx.x, tid = threadIdx.x;
     const int n = n_nodes[b];
     __shared__ unsigned long long s_red[8];
-    __shared__ int32_t s_target[CB_MAX_T];
+    __shared__ int32_t s_target[CB_MAX_T], s_tok[CB_MAX_T], s_par[CB_MAX_T], s_dep[CB_MAX_T];
     __shared__ int s_last;
     if (i < n) {
         const int v0 = ck * chunk, v1 = min(V, v0 + chunk);
@@ -178,10 +176,14 @@ __global__ void __launch_bounds__(256) cb_accept_logits_kernel(
         }
         s_target[k] = tg;
         if (target_out) target_out[(size_t)b * T + k] = tg;
+        // the tree's rows come along, so that the climb from each node to the root below reads shared memory
+        s_tok[k] = k < n ? tok[(size_t)b * T + k] : -1;
+        s_par[k] = k < n ? par[(size_t)b * T + k] : -1;
+        s_dep[k] = k < n ? dep[(size_t)b * T + k] : -1;
     }
     if (tid == 0) ticket[b] = 0u;
     __syncthreads();
-    if (tid < 32) accept_walk(b, T, Dmax, tok, par, dep, n, s_target, n_accept, accept_nodes, out_tokens, tid);
+    if (tid < 32) accept_walk(b, Dmax, s_tok, s_par, s_dep, n, s_target, n_accept, accept_nodes, out_tokens, tid);
 }
 
 __global__ void __launch_bounds__(128) cb_accept_ids_kernel(int B, int T, int Dmax, const int32_t* __restrict__ target_in,
@@ -201,7 +203,7 @@ __global__ void __launch_bounds__(128) cb_accept_ids_kernel(int B, int T, int Dm
         if (target_out) target_out[(size_t)b * T + k] = tg;
     }
     __syncwarp();
-    accept_walk(b, T, Dmax, tok, par, dep, n, s_target[w], n_accept, accept_nodes, out_tokens, lane);
+    accept_walk(b, Dmax, tok + (size_t)b * T, par + (size_t)b * T, dep + (size_t)b * T, n, s_target[w], n_accept, accept_nodes, out_tokens, lane);
 }
 
 }  // namespace
