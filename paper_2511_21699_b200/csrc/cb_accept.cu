@@ -86,7 +86,10 @@ __global__ void __launch_bounds__(256) cb_accept_logits_kernel(
     int32_t* __restrict__ target_out) {
     CB_PDL_ENTRY();
     const int b = blockIdx.z, i = blockIdx.y, ck = blockIdx.x, tid = threadIdx.x;
-    const int n = n_nodes[b];
+    const int n = min(max(n_nodes[b], 0), T);
+    // Rows past the tree have nothing to add and do not queue for the ticket either (hundreds of atomics on one word at
+    // batch 1); an empty tree keeps row 0's CTAs, one of which writes the empty result.
+    if (i >= max(n, 1)) return;
     __shared__ unsigned long long s_red[8];
     __shared__ int32_t s_target[CB_MAX_T], s_tok[CB_MAX_T], s_par[CB_MAX_T], s_dep[CB_MAX_T];
     __shared__ int s_last;
@@ -162,7 +165,7 @@ __global__ void __launch_bounds__(256) cb_accept_logits_kernel(
     // The last CTA of this sequence to arrive owns the walk (and re-zeroes the scratch for the next call).
     if (tid == 0) {
         __threadfence();
-        const uint32_t total = gridDim.x * gridDim.y;
+        const uint32_t total = gridDim.x * (uint32_t)max(n, 1);
         s_last = (atomicAdd(&ticket[b], 1u) == total - 1u) ? 1 : 0;
     }
     __syncthreads();
