@@ -123,6 +123,19 @@ def reduce_over_ranks(seconds, units, device):
     return float(t.item()), float(u.item())
 
 
+def ancestor_masks(par):
+    """Bit-packed ancestor-or-self rows for synthetic full trees given as parent arrays [B, T] (an input of the
+    attention-only shape; drafted trees get their masks from cb_draft_tree)."""
+    B, T = par.shape
+    m = np.zeros((B, T, (T + 31) // 32), np.uint32)
+    for b in range(B):
+        for i in range(T):
+            if par[b, i] >= 0:
+                m[b, i] = m[b, par[b, i]]
+            m[b, i, i // 32] |= np.uint32(1) << np.uint32(i % 32)
+    return m
+
+
 def attn_bytes(cfg, ctx, n_nodes):
     """Algorithmic HBM bytes of one cb_tree_attn launch: cached K and V once, tree K/V, Q in, O out."""
     D, Hkv, Hq = cfg.head_dim, cfg.n_kv_heads, cfg.n_q_heads
@@ -303,7 +316,7 @@ def run_ours(args, rank, world, local_rank):
     if args.full_trees:
         rtrees = [W.random_tree(cfg.seed, b, T, cfg.max_depth, T) for b in range(B)]
         par, dep = np.stack([t[0] for t in rtrees]), np.stack([t[1] for t in rtrees])
-        mask = np.stack([W.tree_mask_from_parents(par[b], T, (T + 31) // 32) for b in range(B)])
+        mask = ancestor_masks(par)
         nn = np.full(B, T, np.int32)
         ftree = dict(tokens=dev(np.maximum(par, 0)), parent=dev(par), depth=dev(dep), mask=dev(mask.view(np.int32)),
                      n_nodes=dev(nn))

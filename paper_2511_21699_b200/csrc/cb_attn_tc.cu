@@ -923,26 +923,38 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
 
 // Merge pass: block (c, *) looks at the unit that CTA c of the attention kernel started but did not finish,
 // and combines the partials that CTA c and the following CTAs left for it.  One warp per output row.
+// Every block waits for the attention grid before it leaves, also the ones that find nothing to merge: the next kernel
+// in the stream is ordered behind this grid only, so this grid must not end while the attention kernel still runs.
 template <int D>
 __global__ void __launch_bounds__(256) cb_attn_merge_kernel(const CbAttnParams p) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the wait comes below, after the set-up that reads inputs only
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x;
     const long long tot = cb_sched_total(p, lane);
-    if (tot <= 0) return;
-    const long long g0 = cb_range_start(tot, p.nc, c), g1 = cb_range_start(tot, p.nc, c + 1);
-    if (g1 <= g0 || g1 >= tot) return;                        // empty range, or the last range
-    int b;
-    long long pre;
-    cb_sched_locate(p, g1 - 1, lane, &b, &pre);
-    const CbSeqShape s = cb_seq_shape(p, b);
-    const long long off = g1 - 1 - pre;
-    const int vt = s.tiles + s.ov;                            // positions of one unit: padding, then its key tiles
-    const int j = (int)(off / vt);
-    if ((int)(off - (long long)j * vt) == vt - 1) return;     // the unit ends with this range
-    const long long ustart = pre + (long long)j * vt, first_tile = ustart + s.ov;
-    if (first_tile < g0) return;                              // started by an earlier CTA: that CTA's block merges it
-    if (first_tile >= g1) return;                             // only padding so far: the next CTA starts the unit
+    bool nothing = tot <= 0;
+    long long g0 = 0, g1 = 0, pre = 0, ustart = 0;
+    int b = 0, j = 0, vt = 1;
+    CbSeqShape s = {};
+    if (!nothing) {
+        g0 = cb_range_start(tot, p.nc, c); g1 = cb_range_start(tot, p.nc, c + 1);
+        nothing = g1 <= g0 || g1 >= tot;                      // empty range, or the last range
+    }
+    if (!nothing) {
+        cb_sched_locate(p, g1 - 1, lane, &b, &pre);
+        s = cb_seq_shape(p, b);
+        const long long off = g1 - 1 - pre;
+        vt = s.tiles + s.ov;                                  // positions of one unit: padding, then its key tiles
+        j = (int)(off / vt);
+        ustart = pre + (long long)j * vt;
+        const long long first_tile = ustart + s.ov;
+        nothing = (int)(off - (long long)j * vt) == vt - 1    // the unit ends with this range
+                  || first_tile < g0                          // started by an earlier CTA: that CTA's block merges it
+                  || first_tile >= g1;                        // only padding so far: the next CTA starts the unit
+    }
+    if (nothing) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        return;
+    }
     const int c_last = cb_cta_of(tot, p.nc, ustart + vt - 1);
     const int kh = j / s.RG, rg = j % s.RG;
     const int nrt = p.MT == 1 ? 1 : min(2, s.mtn - 2 * rg);
@@ -1066,20 +1078,40 @@ int pick_cluster_size(const CbAttnParams& p, int num_sms) {
     return 0;
 }
 
+// Host state of the launcher, per device and guarded: the opt-in to large dynamic shared memory is a per-device function
+// attribute, and the cluster size chosen for a shape is remembered for the shapes seen last.
+constexpr int kMaxDevices = 64;
+constexpr int kShapeMemo = 8;
+struct ShapeMemo { int key[6]; int cs; };
+std::mutex g_launch_mutex;
+bool g_attr_set[2][kMaxDevices];
+ShapeMemo g_shape_memo[kShapeMemo];
+int g_shape_used = 0, g_shape_next = 0;
+
 template <int D>
-cb_status launch(CbAttnParams p, const TcMaps& maps, cudaStream_t st, int num_sms) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        CB_CUDA(cudaFuncSetAttribute(cb_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<D>::SMEM_ALLOC));
-        attr_set = true;
+cb_status launch(CbAttnParams p, const TcMaps& maps, cudaStream_t st, int num_sms, int device) {
+    {
+        std::lock_guard<std::mutex> lock(g_launch_mutex);
+        const int di = device >= 0 && device < kMaxDevices ? device : -1;
+        if (di < 0 || !g_attr_set[D == 128][di]) {
+            CB_CUDA(cudaFuncSetAttribute(cb_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg<D>::SMEM_ALLOC));
+            if (di >= 0) g_attr_set[D == 128][di] = true;
+        }
+        // the choice depends on the shape only
+        const int key[6] = {p.B, p.Hkv, p.MT, num_sms, p.max_tiles, D * kMaxDevices + (di < 0 ? 0 : di)};
+        int found = -1;
+        for (int i = 0; i < g_shape_used && found < 0; ++i) {
+            bool same = true;
+            for (int k = 0; k < 6; ++k) same = same && g_shape_memo[i].key[k] == key[k];
+            if (same) found = i;
+        }
+        if (found < 0) {
+            found = g_shape_used < kShapeMemo ? g_shape_used++ : (g_shape_next++ % kShapeMemo);
+            for (int k = 0; k < 6; ++k) g_shape_memo[found].key[k] = key[k];
+            g_shape_memo[found].cs = pick_cluster_size<D>(p, num_sms);
+        }
+        p.cs = g_shape_memo[found].cs;
     }
-    // the choice depends on the shape only: remember it for the shapes seen last
-    static int memo_key[5] = {-1, -1, -1, -1, -1}, memo_cs = 0;
-    if (memo_key[0] != p.B || memo_key[1] != p.Hkv || memo_key[2] != p.MT || memo_key[3] != num_sms || memo_key[4] != p.max_tiles) {
-        memo_cs = pick_cluster_size<D>(p, num_sms);
-        memo_key[0] = p.B; memo_key[1] = p.Hkv; memo_key[2] = p.MT; memo_key[3] = num_sms; memo_key[4] = p.max_tiles;
-    }
-    p.cs = memo_cs;
     if (p.cs > 0) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(p.B * p.Hkv * p.cs)); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = Cfg<D>::SMEM_ALLOC; cfg.stream = st;
@@ -1141,5 +1173,5 @@ cb_status cb_attn_launch_tensor(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t
         g_map_keys[slot] = key;
         g_map_vals[slot] = maps;
     }
-    return p.D == 128 ? launch<128>(p, maps, st, ctx->num_sms) : launch<64>(p, maps, st, ctx->num_sms);
+    return p.D == 128 ? launch<128>(p, maps, st, ctx->num_sms, ctx->device) : launch<64>(p, maps, st, ctx->num_sms, ctx->device);
 }

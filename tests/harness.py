@@ -15,6 +15,18 @@ def dev(x, dtype=None):
     return t.cuda()
 
 
+def tree_mask_from_parents(par, n, words):
+    """uint32 [T, words]: bit j of row i set iff node j is node i or one of its ancestors; rows >= n zero.  Test input for
+    attention-only cases (synthetic trees); pinned against the oracle's mask routine in test_oracle_attn.py."""
+    T = par.shape[0]
+    m = np.zeros((T, words), dtype=np.uint32)
+    for i in range(n):
+        if par[i] >= 0:
+            m[i] = m[par[i]]
+        m[i, i // 32] |= np.uint32(1) << np.uint32(i % 32)
+    return m
+
+
 class Problem:
     """Streams, contexts and block tables of one config (host side)."""
 
@@ -54,7 +66,7 @@ def synthetic_trees(cfg, full=True):
         if b == 1 and not full:
             n[b] = 1
         par[b], dep[b] = W.random_tree(cfg.seed, b, int(n[b]), cfg.max_depth, T)
-        mask[b] = W.tree_mask_from_parents(par[b], int(n[b]), Wd)
+        mask[b] = tree_mask_from_parents(par[b], int(n[b]), Wd)
     return par, dep, mask, n
 
 
@@ -77,3 +89,89 @@ def oracle_attn_rows(oracle, cfg, prob, mask, b, rows_hi):
 
 def bf16_to_f64(t):
     return t.float().cpu().numpy().astype(np.float64)
+
+
+def oracle_attn_rows_by_head(oracle, cfg, prob, mask, rows, threads=None):
+    """Oracle outputs for rows (b, h, i) anywhere in the batch.  Rows are grouped by (sequence, kv head); each group gets a
+    compact host copy of that head's keys and values only (one kv head, the group's G query heads), so that the full-size
+    configurations stay affordable.  The oracle itself is single-threaded; independent groups run on a thread pool.
+    Returns (out float64 [n, D], lse float64 [n]) in the order of `rows`."""
+    import os
+    from concurrent.futures import ThreadPoolExecutor
+    rows = np.asarray(rows, dtype=np.int64).reshape(-1, 3)
+    P, D, T, G = cfg.page_size, cfg.head_dim, cfg.max_nodes, cfg.gqa
+    groups = {}
+    for r, (b, h, i) in enumerate(rows):
+        groups.setdefault((int(b), int(h) // G), []).append(r)
+    out = np.empty((len(rows), D), np.float64)
+    lse = np.empty(len(rows), np.float64)
+
+    def work(item):
+        (b, kh), idx = item
+        ctx = int(prob.ctx[b])
+        npg = (ctx + P - 1) // P
+        if npg > 0:
+            kp, vp = W.pool_slice_kv(cfg, prob.bt[b, :npg], kh, npg * P, as_f32=False)
+            kp, vp = kp.reshape(npg, P, 1, D), vp.reshape(npg, P, 1, D)
+        else:
+            kp = vp = np.zeros((1, P, 1, D), np.uint16)
+        q = np.stack([W.queries(cfg, b, kh * G + g, as_f32=False) for g in range(G)], axis=1)[None]   # [1, T, G, D]
+        kt, vt = W.tree_kv(cfg, b, kh, as_f32=False)
+        sub = np.array([(0, int(rows[r, 1]) % G, int(rows[r, 2])) for r in idx], np.int32)
+        # long groups are cut into pieces so that the pool keeps all threads busy
+        o, l = oracle.tree_attn_rows(q, kp, vp, np.arange(max(npg, 1), dtype=np.int32)[None], prob.ctx[b:b + 1],
+                                     kt[None, :, None, :], vt[None, :, None, :], mask[b:b + 1], sub)
+        return idx, o, l
+
+    items = []
+    for key, idx in groups.items():
+        step = 256
+        for k in range(0, len(idx), step):
+            items.append((key, idx[k:k + step]))
+    nthreads = threads or min(32, os.cpu_count() or 1)
+    with ThreadPoolExecutor(max_workers=nthreads) as ex:
+        for idx, o, l in ex.map(work, items):
+            out[idx] = o
+            lse[idx] = l
+    return out, lse
+
+
+def shared_unit_rows(cfg, ctx, n, n_ctas, seed=11):
+    """One (b, h, i) row in every unit of tree attention that two persistent CTAs share.
+
+    Restates the decomposition the attention kernel documents: work is counted in 128-key tiles; sequence b has
+    ceil(ctx_b / 128) + 1 of them (the last holds the tree's own keys); a row tile packs 128 / G nodes with the G query
+    heads of a kv head; a unit is one (sequence, kv head, row group), a row group being a pair of row tiles (one when the
+    whole tree cap fits one); every unit is preceded by 3 padding positions when its sequence has two or more row tiles,
+    else 2; all units laid end to end in (sequence, kv head, row group) order are cut into n_ctas equal ranges,
+    range c = [total * c // n_ctas, total * (c + 1) // n_ctas)."""
+    G, Hkv, T = cfg.gqa, cfg.n_kv_heads, cfg.max_nodes
+    npt = 128 // G
+    MT = -(-T // npt)
+    rng = np.random.default_rng(seed)
+    units = []                                             # (first position, padding, tiles, b, kh, rg, row tiles)
+    pos = 0
+    for b in range(cfg.batch):
+        nb = int(min(max(n[b], 0), T))
+        tiles = -(-int(ctx[b]) // 128) + 1
+        mtn = -(-nb // npt)
+        RG = (1 if mtn > 0 else 0) if MT == 1 else (mtn + 1) // 2
+        ov = 3 if mtn >= 2 else 2
+        for kh in range(Hkv):
+            for rg in range(RG):
+                nrt = 1 if MT == 1 else min(2, mtn - 2 * rg)
+                units.append((pos, ov, tiles, b, kh, rg, nrt))
+                pos += ov + tiles
+    total = pos
+    starts = sorted({total * c // n_ctas for c in range(1, n_ctas)})
+    rows, k = [], 0
+    for g in starts:
+        while k + 1 < len(units) and units[k + 1][0] <= g:
+            k += 1
+        p0, ov, tiles, b, kh, rg, nrt = units[k]
+        first, end = p0 + ov, p0 + ov + tiles
+        if first < g < end:                                # key tiles on both sides of the cut
+            rt = rg * 2 + int(rng.integers(0, nrt))
+            lo, hi = rt * npt, min((rt + 1) * npt, int(n[b]))
+            rows.append((b, kh * G + int(rng.integers(0, G)), int(rng.integers(lo, hi))))
+    return rows

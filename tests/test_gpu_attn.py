@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import workloads as W
-from tests.harness import Problem, dev, device_attn_inputs, synthetic_trees, oracle_attn_rows, bf16_to_f64
+from tests.harness import tree_mask_from_parents, Problem, dev, device_attn_inputs, synthetic_trees, oracle_attn_rows, bf16_to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -185,7 +185,7 @@ def test_attn_long_units_mixed_row_tiles_repeated(oracle):
     n[::3] = np.minimum(n[::3], 12)                       # every third tree fits one row tile (16 nodes with 8 heads per group)
     for b in range(0, B, 3):
         par[b], dep[b] = W.random_tree(cfg.seed, b, int(n[b]), cfg.max_depth, T)
-        mask[b] = W.tree_mask_from_parents(par[b], int(n[b]), (T + 31) // 32)
+        mask[b] = tree_mask_from_parents(par[b], int(n[b]), (T + 31) // 32)
     d = device_attn_inputs(cfg, prob)
     cb = Cacheback.from_config(cfg)
     lse = torch.zeros((B, cfg.n_q_heads, T), dtype=torch.float32, device="cuda")

@@ -8,6 +8,7 @@ import torch
 import workloads as W
 from workloads.tensors import pool_full_bits, full_bits, TID
 from workloads.rng import bf16_bits_to_f32
+from tests.harness import tree_mask_from_parents
 
 
 def _setup(cfg, ctx, seed_tree=0, chain=False, star=False):
@@ -27,7 +28,7 @@ def _setup(cfg, ctx, seed_tree=0, chain=False, star=False):
             par = np.zeros(T, dtype=np.int32); par[0] = -1
         else:
             par, _ = W.random_tree(seed_tree, b, n, cfg.max_depth, T)
-        masks.append(W.tree_mask_from_parents(par, n, (T + 31) // 32))
+        masks.append(tree_mask_from_parents(par, n, (T + 31) // 32))
         ns.append(n); pars.append(par)
     return dict(q=q, kp=kp, vp=vp, bt=bt, ctx=ctx, kt=kt, vt=vt, mask=np.stack(masks), n=ns, par=pars)
 
@@ -152,4 +153,44 @@ def test_page_permutation_invariance(oracle):
 
 def test_mask_from_parents_matches_generator(oracle):
     par, _ = W.random_tree(3, 0, 50, 7, 64)
-    assert np.array_equal(oracle.tree_mask(par, 50, 64), W.tree_mask_from_parents(par, 50, 2))
+    assert np.array_equal(oracle.tree_mask(par, 50, 64), tree_mask_from_parents(par, 50, 2))
+
+
+def test_grouped_row_helper_matches_whole_tensor_call(oracle):
+    """The full-size GPU tests call the oracle on one kv head at a time (compact copies of that head's keys); that route
+    must give exactly what the whole-tensor call gives."""
+    from tests.harness import Problem, synthetic_trees, oracle_attn_rows, oracle_attn_rows_by_head
+    cfg = W.CbConfig("attn_small_gqa", 3, 2, 2, 64, 2, 40, 6, 0, 8, 2, 64, (0, 300), 100, 1.1, 0.3, (4, 8), 64)
+    prob = Problem(cfg)
+    par, dep, mask, n = synthetic_trees(cfg, full=False)
+    rng = np.random.default_rng(3)
+    rows = [(int(b), int(rng.integers(0, cfg.n_q_heads)), int(rng.integers(0, n[b]))) for b in rng.integers(0, cfg.batch, 40)]
+    got, got_lse = oracle_attn_rows_by_head(oracle, cfg, prob, mask, rows, threads=3)
+    for k, (b, h, i) in enumerate(rows):
+        ref, ref_lse = oracle_attn_rows(oracle, cfg, prob, mask, b, [(h, i)])
+        assert np.array_equal(got[k], ref[0]) and got_lse[k] == ref_lse[0]
+
+
+def test_shared_unit_rows_lie_in_units_cut_by_a_range_boundary():
+    from tests.harness import shared_unit_rows
+    cfg = W.get_config("c3_8b_gqa")
+    ctx = W.ctx_lens(cfg)
+    n = np.full(cfg.batch, cfg.max_nodes, np.int32)
+    rows = shared_unit_rows(cfg, ctx, n, 148)
+    assert 74 <= len(rows) <= 147
+    # brute force: label every position of the global sequence with its unit and whether it is a key tile
+    G, npt = cfg.gqa, 128 // cfg.gqa
+    label = []
+    for b in range(cfg.batch):
+        tiles = -(-int(ctx[b]) // 128) + 1
+        for kh in range(cfg.n_kv_heads):
+            for rg in range(1):                            # 64 nodes x 4 heads = two row tiles = one row group
+                label += [(b, kh, False)] * 3 + [(b, kh, True)] * tiles
+    total = len(label)
+    cut_units = set()
+    for c in range(1, 148):
+        g = total * c // 148
+        if label[g - 1][:2] == label[g][:2] and label[g - 1][2] and label[g][2]:
+            cut_units.add(label[g][:2])
+    assert {(b, h // G) for b, h, i in rows} == cut_units
+    assert all(0 <= i < cfg.max_nodes for _, _, i in rows)

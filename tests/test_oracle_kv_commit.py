@@ -7,6 +7,7 @@ a K/V swap breaks it; (2) a brute-force element loop on a tiny case; (3) nothing
 import numpy as np
 
 import workloads as W
+from tests.harness import tree_mask_from_parents
 from workloads.tensors import TID
 
 
@@ -22,7 +23,7 @@ def _case(seed, B=3, T=12, Hq=4, Hkv=2, D=64, P=16, ctxs=(5, 16, 37), max_pages=
     par = np.full((B, T), -1, np.int32); dep = np.full((B, T), -1, np.int32); mask = np.zeros((B, T, 1), np.uint32)
     for b in range(B):
         par[b], dep[b] = W.random_tree(seed, b, T, 5, T)
-        mask[b] = W.tree_mask_from_parents(par[b], T, 1)
+        mask[b] = tree_mask_from_parents(par[b], T, 1)
     return dict(bt=bt, ctx=np.array(ctxs, np.int32), kp=kp, vp=vp, kt=kt, vt=vt, q=q, par=par, dep=dep, mask=mask, P=P)
 
 

@@ -8,13 +8,13 @@ fill kernel in ``workloads/fill.cu`` implements the same integer arithmetic).
 from .rng import mix64, normal_i32, normal_f32, normal_bf16_bits, bf16_bits_to_f32, f32_to_bf16_bits, uniform_f64
 from .configs import CbConfig, CONFIGS, get_config
 from .streams import make_stream, make_streams
-from .trees import random_tree, tree_mask_from_parents
+from .trees import random_tree
 from .tensors import (TID, make_block_table, ctx_lens, pool_slice_kv, pool_pages_bits, pool_full_bits, seq_bits,
                       full_bits, tree_kv, queries, logits_rows, plant_logits)
 
 __all__ = [
     "mix64", "normal_i32", "normal_f32", "normal_bf16_bits", "bf16_bits_to_f32", "f32_to_bf16_bits",
     "uniform_f64", "CbConfig", "CONFIGS", "get_config", "make_stream", "make_streams", "random_tree",
-    "tree_mask_from_parents", "TID", "make_block_table", "ctx_lens", "pool_slice_kv", "tree_kv", "queries",
+    "TID", "make_block_table", "ctx_lens", "pool_slice_kv", "tree_kv", "queries",
     "logits_rows", "plant_logits", "pool_pages_bits", "pool_full_bits", "seq_bits", "full_bits",
 ]

@@ -2,8 +2,8 @@
 
 The drafter's real trees depend on the table contents; these stand-ins have exactly ``n`` nodes with
 seeded random parents under a depth cap, parents always preceding children (the order a breadth-first
-drafter emits).  The bit-packed ancestor relation is produced here only as an *input* for attention-only
-cases; the drafter's own mask output is checked separately.
+drafter emits).  Only parents and depths are produced here; the ancestor masks that attention-only cases
+need as an input are made by their callers.
 """
 import numpy as np
 
@@ -29,14 +29,3 @@ def random_tree(seed: int, b: int, n: int, max_depth: int, max_nodes: int = None
         par[i] = cand[pick]
         dep[i] = dep[par[i]] + 1
     return par, dep
-
-
-def tree_mask_from_parents(par: np.ndarray, n: int, words: int) -> np.ndarray:
-    """uint32 [T, words]: bit j of row i set iff node j is node i or one of its ancestors; rows >= n zero."""
-    T = par.shape[0]
-    m = np.zeros((T, words), dtype=np.uint32)
-    for i in range(n):
-        if par[i] >= 0:
-            m[i] = m[par[i]]
-        m[i, i // 32] |= np.uint32(1) << np.uint32(i % 32)
-    return m
