@@ -1,17 +1,24 @@
 #!/usr/bin/env python
 """Benchmark of the Cacheback draft-and-verify step on B200.
 
-A step is one pass of the whole hot path over one batch: cb_update (sliding window over the tokens
-accepted by the previous step) -> cb_draft_tree -> cb_tree_attn -> cb_accept (fp32 logits); the first two are
-issued as the library's one-launch form cb_update_draft_tree unless --separate-calls is given.  The default
-workload is the Llama-2-7B-shaped configuration (batch 1, 32 heads, head_dim 128, context 4,096 in 16-token
-pages, tree cap 64).  Inputs are synthetic (seeded generators in workloads/).  Prints ONE JSON line.
+A step is one pass of the whole hot path over one batch: cb_update (sliding window over the tokens accepted by the
+previous step) -> cb_draft_tree -> cb_tree_attn -> cb_accept (fp32 logits); the first two are issued as the library's
+one-launch form cb_update_draft_tree unless --separate-calls is given.  Inputs are synthetic (seeded generators in
+workloads/).  Prints ONE JSON line.
+
+With no --config the headline is the largest configuration (70B-shaped: batch 128, 64/8 heads, context 32,768, trees of
+128 nodes) with synthetic full trees, so that the attention shape is the stated one; the figure with the drafter's own
+trees stands beside it, and `per_config` holds one record for each of the four full-size configurations (7B-shaped
+batch 1, 8B GQA batch 32, 13B batch 64, 70B batch 128).  With --config NAME only that configuration is run.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+--gpus N > 1 outside a torchrun launch starts N ranks itself (one process per GPU); ranks are independent replicas.
 """
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -25,28 +32,34 @@ sys.path.insert(0, ROOT)
 METRIC = "draft_tree_tokens_verified_per_s"
 UNIT = "tokens/s"
 ADVANCE = 4            # tokens each sequence advances per step (a typical accepted run plus the bonus token)
+HEADLINE = "c5_70b_long"
+FULL_SIZE = ["c2_7b", "c3_8b_gqa", "c4_13b_turns", "c5_70b_long"]
 
 
-def parse():
+def parse(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=48)
-    ap.add_argument("--warmup", type=int, default=6)
-    ap.add_argument("--config", default="c2_7b")
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default=None, help="one workload only (default: headline %s plus per_config records)" % HEADLINE)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--full-trees", action="store_true", help="attention/acceptance on synthetic full-size trees")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--drafted-headline", action="store_true", help="headline value from the drafter's own trees instead of full ones")
     ap.add_argument("--separate-calls", action="store_true", help="cb_update and cb_draft_tree as two launches")
     ap.add_argument("--frozen", type=int, default=0, metavar="TOKENS",
                     help="attach a frozen table built on the GPU from a synthetic corpus of this many tokens (0 = none)")
-    return ap.parse_args()
+    ap.add_argument("--rank-plumbing-only", action="store_true", help=argparse.SUPPRESS)
+    return ap.parse_args(argv)
 
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one cb_attn_tc_kernel launch, from the ncu capture
-# summarised in profiles/cb_attn_tc_kernel_<workload>.md.  It is reported only while the kernel sources still hash to the
-# captured ones; after any change to them the figure is stale and `traffic` is null until the capture is redone.
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one cb_attn_tc_kernel launch with full trees, from the ncu
+# captures summarised under profiles/.  Reported only while the kernel sources still hash to the captured ones; after any
+# change to them the figure is stale and `traffic` is null until the capture is redone.
 ATTN_TRAFFIC = {"sources_sha1": "940d4a8002e5bcb4876bd7445ef665e14f2a13aa",
-                "bytes_per_launch": {"c2_7b": 70.37e6, "c3_8b_gqa": 558.2e6, "c4_13b_turns": 2768.5e6}}
+                "bytes_per_launch": {"c2_7b": 70.37e6, "c3_8b_gqa": 558.2e6, "c4_13b_turns": 2768.5e6},
+                "source": {"c2_7b": "profiles/cb_attn_tc_kernel_c2_7b.md", "c3_8b_gqa": "profiles/cb_attn_tc_kernel_c3_c4.md",
+                           "c4_13b_turns": "profiles/cb_attn_tc_kernel_c3_c4.md"}}
 
 
 def attn_sources_sha1():
@@ -63,8 +76,9 @@ def peaks():
     if os.path.exists(p):
         with open(p) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured"
-    return 6650.0, 1590.0, "fallback"
+        return {"hbm_gbs": float(d["hbm_gbs"]), "tflops": float(d["bf16_tflops"]),
+                "tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "kind": "measured (MEASURED_PEAKS.json)"}
+    return {"hbm_gbs": 6650.0, "tflops": 1590.0, "tflops_sustained": 1400.0, "kind": "fallback"}
 
 
 class ClockSampler:
@@ -123,6 +137,20 @@ def reduce_over_ranks(seconds, units, device):
     return float(t.item()), float(u.item())
 
 
+def free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(n, argv):
+    """Starts this script as n ranks of one node (one process per GPU) and passes their output through; used when
+    --gpus n > 1 is given outside a torchrun launch."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n), "--master-addr", "127.0.0.1",
+           "--master-port", str(free_port()), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
 def ancestor_masks(par):
     """Bit-packed ancestor-or-self rows for synthetic full trees given as parent arrays [B, T] (an input of the
     attention-only shape; drafted trees get their masks from cb_draft_tree)."""
@@ -143,128 +171,125 @@ def attn_bytes(cfg, ctx, n_nodes):
 
 
 def attn_flops(cfg, ctx, n_nodes, pairs):
+    """4 * Hq * D * (node-context pairs + node-ancestor pairs): the two products of attention."""
     return float(4.0 * cfg.n_q_heads * cfg.head_dim * (np.sum(n_nodes * ctx.astype(np.float64)) + pairs))
 
 
-# --------------------------------------------------------------------------------------------------------
-def run_reference(args, rank, world):
-    """The oracle, as it stands, timed on the host cores (single thread) on a bounded sample of the step."""
-    if rank != 0:
-        return
-    import workloads as W
-    from workloads.tensors import TID
-    from oracle import cb_oracle as orc
-    cfg = W.get_config(args.config)
-    ctx = W.ctx_lens(cfg)
-    toks, lens = W.make_streams(cfg, ctx)
-    bt, num_pages = W.make_block_table(cfg, ctx)
-    B, T = cfg.batch, cfg.max_nodes
-    nb = min(B, 2)                                         # sequences per sampled step
-    nh = min(cfg.n_q_heads, 4)                             # attention heads per sampled step
-    tabs = [orc.OracleTable(cfg.LL, cfg.FL, cfg.LC, cfg.FC) for _ in range(nb)]
-    pos = np.minimum(ctx + 1, lens)[:nb].astype(np.int64)
-    for b in range(nb):
-        tabs[b].update(toks[b], 0, int(pos[b]))
-    kv = {}
-    for b in range(nb):
-        npg = (int(ctx[b]) + cfg.page_size - 1) // cfg.page_size
-        kp, vp = W.pool_pages_bits(cfg, bt[b, :npg])
-        kv[b] = (kp, vp, W.seq_bits(cfg, TID.Q, b, cfg.n_q_heads)[None], W.seq_bits(cfg, TID.K_TREE, b, cfg.n_kv_heads)[None],
-                 W.seq_bits(cfg, TID.V_TREE, b, cfg.n_kv_heads)[None], np.arange(npg, dtype=np.int32)[None])
-    steps = max(1, min(args.steps, 8))
-    warm = min(args.warmup, 1)
-    t_total, tok_total = 0.0, 0
-    for s in range(warm + steps):
-        t_step, n_step = 0.0, 0
-        for b in range(nb):
-            t0 = time.perf_counter()
-            tabs[b].update(toks[b], int(pos[b]), int(pos[b]) + ADVANCE)
-            pos[b] += ADVANCE
-            n, tok, par, dep, mask = tabs[b].draft_tree(toks[b], int(pos[b]), T, cfg.crt, cfg.max_depth)
-            t1 = time.perf_counter()
-            kp, vp, q, kt, vt, btl = kv[b]
-            rows = np.array([(0, h, i) for h in range(nh) for i in range(n)], np.int32)
-            orc.tree_attn_rows(q, kp, vp, btl, ctx[b:b + 1], kt, vt, mask[None], rows)
-            t2 = time.perf_counter()
-            lr = W.logits_rows(cfg, b, np.arange(n))
-            t3 = time.perf_counter()
-            tgt = np.full(T, -1, np.int32)
-            tgt[:n] = orc.argmax_rows(lr)
-            orc.accept(tok, par, dep, n, tgt, cfg.max_depth)
-            t4 = time.perf_counter()
-            # attention is sampled on nh of Hq heads: scale its time to all heads; logits generation (t2..t3) is input
-            # preparation and is not counted
-            t_step += (t1 - t0) + (t2 - t1) * (cfg.n_q_heads / nh) + (t4 - t3)
-            n_step += n
-        if s >= warm:
-            t_total += t_step * (B / nb)                   # one thread walks the batch sequence by sequence
-            tok_total += n_step * (B / nb)
-    val = tok_total / t_total
-    sample = ("%d of %d sequences, %d of %d q heads per step (attention time scaled by heads, step time by sequences), "
-              "%d steps, single thread" % (nb, B, nh, cfg.n_q_heads, steps))
-    print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps, "warmup": warm,
-        "ms_per_step": 1e3 * t_total / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64", "data": "synthetic", "config": {"workload": cfg.name, "batch": B, "tree_cap": T},
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
-        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+def attn_roofline(cfg, ctx, n_nodes, pairs, ms, pk):
+    """Roofline record of one cb_tree_attn launch (attention kernel plus its merge pass): the slower of bytes over the
+    measured copy bandwidth and flops over the measured bf16 matmul rate."""
+    a_bytes, fl = attn_bytes(cfg, ctx, n_nodes), attn_flops(cfg, ctx, n_nodes, pairs)
+    t_mem, t_cmp = a_bytes / (pk["hbm_gbs"] * 1e9), fl / (pk["tflops"] * 1e12)
+    if t_mem >= t_cmp:
+        r = {"bound": "hbm", "achieved": a_bytes / (ms * 1e-3) / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s"}
+    else:
+        r = {"bound": "tensor", "achieved": fl / (ms * 1e-3) / 1e12, "peak": pk["tflops"], "unit": "TFLOP/s"}
+        r["frac_of_sustained"] = r["achieved"] / pk["tflops_sustained"]
+        r["peak_sustained"] = pk["tflops_sustained"]
+    r["frac"] = r["achieved"] / r["peak"]
+    r.update({"ms_per_launch": ms, "algorithmic_bytes": a_bytes, "flops": fl, "gbs": a_bytes / (ms * 1e-3) / 1e9,
+              "tflops": fl / (ms * 1e-3) / 1e12, "roofline_ms": 1e3 * max(t_mem, t_cmp), "peak_source": pk["kind"]})
+    return r
 
 
 # --------------------------------------------------------------------------------------------------------
-def cpu_baseline(cfg, prob_host, tree_host):
-    """Oracle timed on this machine's host cores on a bounded sample of the same workload (rank 0, N = 1)."""
+def oracle_sample(cfg, ctx, toks, lens, bt, steps, full_trees, nb=2, nh=2, nn=16):
+    """The oracle, as it stands, timed single-threaded on a bounded sample of the step: nb sequences; table update,
+    drafting, arg-max and acceptance whole; attention on nh query heads and (with full trees) nn of the tree's nodes,
+    its time scaled to all heads and nodes.  Returns (tokens per step of the whole batch, seconds per step of the whole
+    batch, words describing the sample)."""
     import workloads as W
-    from workloads.tensors import TID
     from oracle import cb_oracle as orc
-    ctx, toks, lens, bt = prob_host
     B, T = cfg.batch, cfg.max_nodes
-    nb, nh = min(B, 2), min(cfg.n_q_heads, 4)
-    t_step, n_tok = 0.0, 0
+    nb, nh = min(B, nb), min(cfg.n_q_heads, nh)
+    G = cfg.gqa
+    t_total, tok_total = 0.0, 0.0
     for b in range(nb):
         tab = orc.OracleTable(cfg.LL, cfg.FL, cfg.LC, cfg.FC)
         pos = int(min(ctx[b] + 1, lens[b]))
         tab.update(toks[b], 0, pos)
         npg = (int(ctx[b]) + cfg.page_size - 1) // cfg.page_size
-        kp, vp = W.pool_pages_bits(cfg, bt[b, :npg])
-        q = W.seq_bits(cfg, TID.Q, b, cfg.n_q_heads)[None]
-        kt = W.seq_bits(cfg, TID.K_TREE, b, cfg.n_kv_heads)[None]
-        vt = W.seq_bits(cfg, TID.V_TREE, b, cfg.n_kv_heads)[None]
-        for rep in range(2):
+        heads = list(range(nh))
+        kvs = {}
+        for kh in sorted({h // G for h in heads}):          # the sampled heads' kv heads only: one compact copy per kv head
+            kp, vp = W.pool_slice_kv(cfg, bt[b, :npg], kh, npg * cfg.page_size, as_f32=False)
+            kt, vt = W.tree_kv(cfg, b, kh, as_f32=False)
+            kvs[kh] = (kp.reshape(npg, cfg.page_size, 1, cfg.head_dim), vp.reshape(npg, cfg.page_size, 1, cfg.head_dim),
+                       kt[None, :, None, :], vt[None, :, None, :])
+        qh = {h: W.queries(cfg, b, h, as_f32=False)[None, :, None, :] for h in heads}
+        if full_trees:
+            fpar, fdep = W.random_tree(cfg.seed, b, T, cfg.max_depth, T)
+            fmask = orc.tree_mask(fpar, T, T)
+        for rep in range(steps):
             t0 = time.perf_counter()
             tab.update(toks[b], pos, pos + ADVANCE)
             pos += ADVANCE
             n, tok, par, dep, mask = tab.draft_tree(toks[b], pos, T, cfg.crt, cfg.max_depth)
             t1 = time.perf_counter()
-            rows = np.array([(0, h, i) for h in range(nh) for i in range(n)], np.int32)
-            orc.tree_attn_rows(q, kp, vp, np.arange(npg, dtype=np.int32)[None], ctx[b:b + 1], kt, vt, mask[None], rows)
+            if full_trees:
+                n, par, dep, mask, tok = T, fpar, fdep, fmask, np.maximum(fpar, 0).astype(np.int32)
+            nodes = list(range(n))
+            if full_trees and n > nn:
+                nodes = sorted(set(range(0, n, n // nn)))[:nn]
+            rows = np.array([(0, 0, i) for i in nodes], np.int32)
             t2 = time.perf_counter()
-            lr = W.logits_rows(cfg, b, np.arange(n))
+            for h in heads:
+                kp, vp, kt, vt = kvs[h // G]
+                orc.tree_attn_rows(qh[h], kp, vp, np.arange(npg, dtype=np.int32)[None], ctx[b:b + 1], kt, vt, mask[None], rows)
             t3 = time.perf_counter()
+            lr = W.logits_rows(cfg, b, np.arange(n))        # input preparation, not counted
+            t4 = time.perf_counter()
             tgt = np.full(T, -1, np.int32)
             tgt[:n] = orc.argmax_rows(lr)
             orc.accept(tok, par, dep, n, tgt, cfg.max_depth)
-            t4 = time.perf_counter()
-            t_step += (t1 - t0) + (t2 - t1) * (cfg.n_q_heads / nh) + (t4 - t3)
-            n_tok += n
-    return {"value": n_tok / t_step, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": "%d of %d sequences x 2 steps, %d of %d q heads (attention time scaled by heads); single thread"
-                      % (nb, B, nh, cfg.n_q_heads)}
+            t5 = time.perf_counter()
+            t_total += (t1 - t0) + (t3 - t2) * (cfg.n_q_heads / nh) * (n / len(nodes)) + (t5 - t4)
+            tok_total += n
+    per_step_tokens = tok_total / (nb * steps) * B
+    per_step_seconds = t_total / (nb * steps) * B          # one thread walks the batch sequence by sequence
+    sample = ("%d of %d sequences x %d steps; update, draft, arg-max and acceptance whole; attention on %d of %d q heads%s, "
+              "its time scaled by heads%s (an extrapolation by flop count); step time scaled by sequences; single thread"
+              % (nb, B, steps, nh, cfg.n_q_heads, (" and %d of %d nodes" % (min(nn, T), T)) if full_trees else "",
+                 " and nodes" if full_trees else ""))
+    return per_step_tokens, per_step_seconds, sample
 
 
-def run_ours(args, rank, world, local_rank):
+def run_reference(args, rank, world):
+    """The oracle, as it stands, timed on the host cores (single thread) on a bounded sample of the step."""
+    if rank != 0:
+        return
+    import workloads as W
+    cfg = W.get_config(args.config or HEADLINE)
+    ctx = W.ctx_lens(cfg)
+    toks, lens = W.make_streams(cfg, ctx)
+    bt, num_pages = W.make_block_table(cfg, ctx)
+    steps = max(1, min(args.steps, 3))
+    full = not args.drafted_headline
+    tokens, seconds, sample = oracle_sample(cfg, ctx, toks, lens, bt, steps, full)
+    val = tokens / seconds
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps, "warmup": 0,
+        "ms_per_step": 1e3 * seconds, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "batch": cfg.batch, "tree_cap": cfg.max_nodes, "trees": "synthetic full" if full else "drafted"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+# --------------------------------------------------------------------------------------------------------
+def measure(args, cfg_name, rank, world, device, headline):
+    """Everything measured on one configuration.  Returns the record; a headline record also carries the pieces of the
+    top-level line (keys that start with an underscore: whole-job value, end-to-end figure, launch count)."""
     import torch
     import workloads as W
     from workloads import device as wdev
     from workloads.tensors import TID
     from paper_2511_21699_b200 import Cacheback
+    from dataclasses import replace
 
-    torch.cuda.set_device(local_rank)
-    device = torch.device("cuda", local_rank)
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=device)
-    from dataclasses import replace
-    cfg = replace(W.get_config(args.config), seed=rank)        # every rank has its own batch of sequences
+    cfg = replace(W.get_config(cfg_name), seed=rank)        # every rank has its own batch of sequences
     B, T = cfg.batch, cfg.max_nodes
     ctx = W.ctx_lens(cfg)
     toks, lens = W.make_streams(cfg, ctx)
@@ -272,6 +297,7 @@ def run_ours(args, rank, world, local_rank):
     K, Wm = args.steps, max(args.warmup, 3)
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
     bf = torch.bfloat16
+    pk = peaks()
 
     # Rotate through R copies of the streamed tensors so that no step finds its inputs in the 126 MB L2.
     pool_bytes = num_pages * cfg.page_size * cfg.n_kv_heads * cfg.head_dim * 2 * 2
@@ -287,14 +313,48 @@ def run_ours(args, rank, world, local_rank):
     vt = wdev.fill_normal(torch.empty((B, T, cfg.n_kv_heads, cfg.head_dim), dtype=bf, device=device), cfg.seed, TID.V_TREE)
     bt_d, ctx_d, toks_d = dev(bt), dev(ctx), dev(toks)
     out = torch.empty_like(q)
+    max_ctx = int(ctx.max())
 
     cb = Cacheback.from_config(cfg, device=device)
     prefill = np.minimum(ctx + 1, lens).astype(np.int32)
-    total = 2 * (Wm + K) + 4
+    total = 3 * (Wm + K) + 8
     assert int((lens - prefill).min()) > ADVANCE * total + T, "stream too short for this many steps"
     n_old = dev(np.stack([prefill + ADVANCE * s for s in range(total)]).astype(np.int32))
     n_new = dev(np.stack([prefill + ADVANCE * (s + 1) for s in range(total)]).astype(np.int32))
-    cb.cb_update_bulk(toks_d, dev(np.zeros(B, np.int32)), dev(prefill))     # prompt initialisation, untimed
+    zeros_d, prefill_d = dev(np.zeros(B, np.int32)), dev(prefill)
+
+    stream = torch.cuda.Stream(device=device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, reps=3):
+        tt = []
+        for _ in range(reps):
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            stream.synchronize()
+            tt.append(e0.elapsed_time(e1))
+        return float(np.median(tt))
+
+    with torch.cuda.stream(stream):
+        # ---- prompt initialisation (the bulk form of cb_update), timed on its own: the tables start empty each time
+        bulk_ms = []
+        for rep in range(3):
+            cb.cb_reset()
+            stream.synchronize()
+            e0.record(stream)
+            cb.cb_update_bulk(toks_d, zeros_d, prefill_d)
+            e1.record(stream)
+            stream.synchronize()
+            bulk_ms.append(e0.elapsed_time(e1))
+    windows = float(np.sum(np.maximum(prefill.astype(np.int64) - cfg.LL - cfg.FL + 1, 0)))
+    entry_bytes = (cfg.LL + 1 + cfg.FC * (cfg.FL + 1)) * 4
+    bulk_bytes = windows * (entry_bytes + (cfg.FL + 2) * 4)
+    bulk_t = float(np.median(bulk_ms)) * 1e-3
+    bulk = {"ms": 1e3 * bulk_t, "windows": windows, "windows_per_s": windows / bulk_t, "algorithmic_bytes": bulk_bytes,
+            "bytes_per_window": entry_bytes + (cfg.FL + 2) * 4, "gbs": bulk_bytes / bulk_t / 1e9,
+            "frac_of_hbm": bulk_bytes / bulk_t / 1e9 / pk["hbm_gbs"]}
+
     frozen_info = None
     if args.frozen > 0:
         # Stand-in for the paper's corpus sample: streams of the workload's own token distribution under other seeds.
@@ -311,202 +371,270 @@ def run_ours(args, rank, world, local_rank):
         cb.cb_frozen_attach(ft)
         frozen_info = {"corpus_tokens": int(corpus.numel()), "LC": 1 << 16, "FC": min(16, 2 * cfg.FC),
                        "leaders": int(len(ft.cb_frozen_dump()[0])), "build_ms": fe0.elapsed_time(fe1)}
+
     trees = [cb.alloc_tree() for _ in range(total)]         # every step keeps its own tree, so later passes can reuse it
     res = cb.alloc_accept()
-    if args.full_trees:
-        rtrees = [W.random_tree(cfg.seed, b, T, cfg.max_depth, T) for b in range(B)]
-        par, dep = np.stack([t[0] for t in rtrees]), np.stack([t[1] for t in rtrees])
-        mask = ancestor_masks(par)
-        nn = np.full(B, T, np.int32)
-        ftree = dict(tokens=dev(np.maximum(par, 0)), parent=dev(par), depth=dev(dep), mask=dev(mask.view(np.int32)),
-                     n_nodes=dev(nn))
+    rtrees = [W.random_tree(cfg.seed, b, T, cfg.max_depth, T) for b in range(B)]
+    fpar, fdep = np.stack([t[0] for t in rtrees]), np.stack([t[1] for t in rtrees])
+    ftree = dict(tokens=dev(np.maximum(fpar, 0)), parent=dev(fpar), depth=dev(fdep), mask=dev(ancestor_masks(fpar).view(np.int32)),
+                 n_nodes=dev(np.full(B, T, np.int32)))
+    full_pairs = float(np.sum(fdep + 1))                    # node-ancestor pairs of the synthetic full trees (self included)
 
-    def step(s):
-        r = s % R
-        tr = trees[s]
+    def front(s):
         if args.separate_calls:
             cb.cb_update(toks_d, n_old[s], n_new[s])
-            cb.cb_draft_tree(toks_d, n_new[s], tr)
+            cb.cb_draft_tree(toks_d, n_new[s], trees[s])
         else:
-            cb.cb_update_draft_tree(toks_d, n_old[s], n_new[s], tr)
-        at = ftree if args.full_trees else tr
-        cb.cb_tree_attn(q, kps[r], vps[r], bt_d, ctx_d, kt, vt, at["mask"], at["n_nodes"], out=out, max_ctx=int(ctx.max()))
+            cb.cb_update_draft_tree(toks_d, n_old[s], n_new[s], trees[s])
+
+    def step(s, full):
+        r = s % R
+        front(s)
+        at = ftree if full else trees[s]
+        cb.cb_tree_attn(q, kps[r], vps[r], bt_d, ctx_d, kt, vt, at["mask"], at["n_nodes"], out=out, max_ctx=max_ctx)
         cb.cb_accept(at, logits=lgs[r], res=res)
 
-    stream = torch.cuda.Stream(device=device)
+    def one_call(which, s):
+        r = s % R
+        tr = trees[s]
+        if which == "cb_update":
+            cb.cb_update(toks_d, n_old[s], n_new[s])
+        elif which == "cb_draft_tree":
+            cb.cb_draft_tree(toks_d, n_new[s], tr)
+        elif which == "cb_update_draft_tree":
+            cb.cb_update_draft_tree(toks_d, n_old[s], n_new[s], tr)
+        elif which == "cb_tree_attn":
+            cb.cb_tree_attn(q, kps[r], vps[r], bt_d, ctx_d, kt, vt, ftree["mask"], ftree["n_nodes"], out=out, max_ctx=max_ctx)
+        elif which == "cb_tree_attn_drafted":
+            cb.cb_tree_attn(q, kps[r], vps[r], bt_d, ctx_d, kt, vt, tr["mask"], tr["n_nodes"], out=out, max_ctx=max_ctx)
+        elif which == "cb_accept":
+            cb.cb_accept(ftree, logits=lgs[r], res=res)
+        else:
+            cb.cb_accept(tr, logits=lgs[r], res=res)
+
+    rec = {"workload": cfg_name}
     with torch.cuda.stream(stream):
         for s in range(Wm):                                  # eager warm-up (also sets kernel attributes)
-            step(s)
+            step(s, s % 2 == 0)
         stream.synchronize()
-        # The K timed steps are captured once into a CUDA graph: at batch 1 a step is a handful of
-        # microsecond-scale kernels and host launch cost would otherwise dominate.
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g, stream=stream):
-            for s in range(Wm, Wm + K):
-                step(s)
+        # The K timed steps are captured once into a CUDA graph: at batch 1 a step is a handful of microsecond-scale
+        # kernels and host launch cost would otherwise dominate.  The two graphs (full trees, drafted trees) walk
+        # disjoint step indices of the token streams.
+        graphs = {}
+        for full, base in ((True, Wm), (False, Wm + K)):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for s in range(base, base + K):
+                    step(s, full)
+            graphs[full] = g
         launches0 = cb.launch_count()
         for s in range(Wm, Wm + K):                          # same sequence eagerly, to count launches
-            step(s)
+            step(s, True)
         launches = cb.launch_count() - launches0
         stream.synchronize()
         if world > 1:
             dist.barrier()
-        sampler = ClockSampler(local_rank)
+        sampler = ClockSampler(device.index or 0)
         sampler.start()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
-        times = []
-        reps = 3
-        while len(times) < reps:
-            e0.record(stream)
-            g.replay()
-            e1.record(stream)
-            stream.synchronize()
-            times.append(e0.elapsed_time(e1))
-            if len(times) == 3:
-                # keep replaying until the timed region spans about 0.4 s, so that the clock sampler sees it
-                reps = int(min(400, max(3, 400.0 / max(float(np.median(times)), 1e-3))))
-        ms_total = float(np.median(times))
-        nn_timed = torch.stack([t["n_nodes"] for t in trees[Wm:Wm + K]]).cpu().numpy().astype(np.float64)
-        # Per-call times, for the roofline of the dominant kernel: each of the four calls is captured K times back to
-        # back in a graph of its own (inputs rotating as in the step) and the replay is timed with events on this stream.
-        # Eager launches would measure the host's enqueue cost at batch 1, not the kernels.
-        base = Wm + K
-
-        def one_call(which, s):
-            r = s % R
-            tr = trees[s]
-            at = ftree if args.full_trees else tr
-            if which == 0:
-                cb.cb_update(toks_d, n_old[s], n_new[s])
-            elif which == 1:
-                cb.cb_draft_tree(toks_d, n_new[s], tr)
-            elif which == 2:
-                cb.cb_tree_attn(q, kps[r], vps[r], bt_d, ctx_d, kt, vt, at["mask"], at["n_nodes"], out=out, max_ctx=int(ctx.max()))
-            elif which == 3:
-                cb.cb_accept(at, logits=lgs[r], res=res)
-            else:
-                cb.cb_update_draft_tree(toks_d, n_old[s], n_new[s], tr)
-
+        step_ms, reps_used = {}, {}
+        for full in (True, False):
+            times = []
+            reps = 3
+            while len(times) < reps:
+                e0.record(stream)
+                graphs[full].replay()
+                e1.record(stream)
+                stream.synchronize()
+                times.append(e0.elapsed_time(e1))
+                if len(times) == 3:
+                    # keep replaying until the timed region spans about 0.4 s, so that the clock sampler sees it
+                    reps = int(min(400, max(3, 400.0 / max(float(np.median(times)), 1e-3))))
+            step_ms[full] = float(np.median(times)) / K
+            reps_used[full] = reps
+        nn_drafted = torch.stack([t["n_nodes"] for t in trees[Wm + K:Wm + 2 * K]]).cpu().numpy().astype(np.float64)
+        # Per-call times, for the roofline of the dominant kernel: each call is captured K times back to back in a graph of
+        # its own (inputs rotating as in the step) and the replay is timed with events on this stream.  Eager launches
+        # would measure the host's enqueue cost at batch 1, not the kernels.
+        base = 2 * (Wm + K)
         for s in range(base, base + K):                      # one eager pass leaves valid trees for every step index
-            step(s)
+            step(s, False)
         stream.synchronize()
-        per_med = np.zeros(5)
-        for which in range(5):
+        per_call = {}
+        for which in ("cb_update", "cb_draft_tree", "cb_update_draft_tree", "cb_tree_attn", "cb_tree_attn_drafted", "cb_accept",
+                      "cb_accept_drafted"):
             gc = torch.cuda.CUDAGraph()
             with torch.cuda.graph(gc, stream=stream):
                 for s in range(base, base + K):
                     one_call(which, s)
-            tt = []
-            for _ in range(3):
-                e0.record(stream)
-                gc.replay()
-                e1.record(stream)
-                stream.synchronize()
-                tt.append(e0.elapsed_time(e1) / K)
-            per_med[which] = float(np.median(tt))
+            per_call[which] = timed(gc.replay) / K
             del gc
         nn_percall = torch.stack([t["n_nodes"] for t in trees[base:base + K]]).cpu().numpy().astype(np.float64)
         clocks = sampler.stop()
-    nn_attn = (np.full((K, B), float(T)) if args.full_trees else nn_timed)
-    if args.full_trees:
-        nn_percall = np.full((K, B), float(T))
-    tokens = float(nn_attn.sum())
-    local_tokens = tokens
-    if world > 1:
-        ms_total, tokens = reduce_over_ranks(ms_total, tokens, device)
-    value = tokens / (ms_total * 1e-3)
+    del graphs
 
-    # end to end through the public API with host buffers: H2D of the step's inputs, D2H of its result
-    pin = lambda t: t.cpu().pin_memory()
-    hq, hkt, hvt, hlg = pin(q), pin(kt), pin(vt), pin(lgs[0])
-    h_old, h_new = pin(n_old), pin(n_new)
-    dq, dkt, dvt, dlg = torch.empty_like(q), torch.empty_like(kt), torch.empty_like(vt), torch.empty_like(lgs[0])
-    d_old, d_new = torch.empty(B, dtype=torch.int32, device=device), torch.empty(B, dtype=torch.int32, device=device)
-    h_acc = torch.empty(B, dtype=torch.int32).pin_memory()
-    h_out = torch.empty(B, cfg.max_depth + 1, dtype=torch.int32).pin_memory()
-    h2d = sum(t.numel() * t.element_size() for t in (hq, hkt, hvt, hlg)) + 2 * B * 4
-    d2h = h_acc.numel() * 4 + h_out.numel() * 4
-    e2e_tokens = 0.0
-    with torch.cuda.stream(stream):
-        def e2e_step(s):
-            r = s % R
-            dq.copy_(hq, non_blocking=True); dkt.copy_(hkt, non_blocking=True); dvt.copy_(hvt, non_blocking=True)
-            dlg.copy_(hlg, non_blocking=True)
-            d_old.copy_(h_old[s], non_blocking=True); d_new.copy_(h_new[s], non_blocking=True)
-            tr = trees[s]
-            if args.separate_calls:
-                cb.cb_update(toks_d, d_old, d_new)
-                cb.cb_draft_tree(toks_d, d_new, tr)
-            else:
-                cb.cb_update_draft_tree(toks_d, d_old, d_new, tr)
-            at = ftree if args.full_trees else tr
-            cb.cb_tree_attn(dq, kps[r], vps[r], bt_d, ctx_d, dkt, dvt, at["mask"], at["n_nodes"], out=out, max_ctx=int(ctx.max()))
-            cb.cb_accept(at, logits=dlg, res=res)
-            h_acc.copy_(res["n_accept"], non_blocking=True); h_out.copy_(res["out_tokens"], non_blocking=True)
-            stream.synchronize()
-        for s in range(Wm, Wm + 3):
-            e2e_step(s)
-        t0 = time.perf_counter()
-        for s in range(Wm, Wm + K):
-            e2e_step(s)
-        e2e_s = time.perf_counter() - t0
-    e2e_tokens = local_tokens
-    if world > 1:
-        e2e_s, e2e_tokens = reduce_over_ranks(e2e_s, local_tokens, device)
-    e2e_val = e2e_tokens / e2e_s
+    nn_full = np.full(B, float(T))
+    nn_mean = nn_percall.mean(axis=0)                        # trees of the steps the per-call graphs ran
+    roof_full = attn_roofline(cfg, ctx, nn_full, full_pairs, per_call["cb_tree_attn"], pk)
+    # the drafter reports no depths here: 4 ancestors per node stand in for the drafted trees' mean
+    roof_drafted = attn_roofline(cfg, ctx, nn_mean, float(np.sum(nn_mean * 4)), per_call["cb_tree_attn_drafted"], pk)
+    traffic, traffic_source = None, "none: no ncu capture of the kernel sources as they are now"
+    if ATTN_TRAFFIC["sources_sha1"] == attn_sources_sha1() and cfg_name in ATTN_TRAFFIC["bytes_per_launch"]:
+        traffic = ATTN_TRAFFIC["bytes_per_launch"][cfg_name]
+        traffic_source = ATTN_TRAFFIC["source"][cfg_name] + " (ncu dram__bytes_read.sum + dram__bytes_write.sum; kernel sources hash-matched)"
+    roof_full.update({"traffic": traffic, "traffic_source": traffic_source,
+                      "kernel": "cb_tree_attn (attention kernel, plus its merge pass where the launch is not in cluster mode)"})
+    acc_bytes_full, acc_bytes_dr = float(B * T) * cfg.vocab * 4, float(np.sum(nn_mean)) * cfg.vocab * 4
+    accept = {"gbs": acc_bytes_full / (per_call["cb_accept"] * 1e-3) / 1e9, "algorithmic_bytes": acc_bytes_full,
+              "ms_per_launch": per_call["cb_accept"],
+              "gbs_drafted_trees": acc_bytes_dr / (per_call["cb_accept_drafted"] * 1e-3) / 1e9}
+    accept["frac_of_hbm"] = accept["gbs"] / pk["hbm_gbs"]
+    accept["frac_of_hbm_drafted_trees"] = accept["gbs_drafted_trees"] / pk["hbm_gbs"]
+    tok_full, tok_dr = float(B * T), float(nn_drafted.sum()) / K
+    rec.update({
+        "batch": B, "tree_cap": T, "context": [int(ctx.min()), int(ctx.max())],
+        "ms_per_step": step_ms[True], "ms_per_step_drafted_trees": step_ms[False],
+        "value_full_trees": tok_full / (step_ms[True] * 1e-3), "value_drafted_trees": tok_dr / (step_ms[False] * 1e-3),
+        "mean_tree_nodes_drafted": float(nn_drafted.mean()),
+        "per_call_ms": per_call, "roofline": roof_full, "roofline_drafted_trees": roof_drafted, "accept": accept,
+        "prompt_ingest": bulk, "clocks": clocks,
+        "l2": "rotating %d copies of K/V pool and logits (%.0f MB)" % (R, R * (pool_bytes + logit_bytes) / 1e6),
+        "replays": reps_used[True]})
+    if B == 1:
+        rec["latency_bound"] = ("at batch 1 cb_update, cb_draft_tree and cb_accept move a few KB to a few MB per call through chains "
+                                "of dependent memory round trips: their time is launch plus round trips, not bandwidth")
 
+    if not headline:
+        st, counters = cb.cb_poll_status()
+        assert st == 0, "device status %d" % st
+        return rec
+
+    # ---- whole-job figures over ranks
+    full = not args.drafted_headline
+    seconds, tokens = step_ms[full] * 1e-3, (tok_full if full else tok_dr)
+    if world > 1:
+        seconds, tokens = reduce_over_ranks(seconds, tokens, device)
+    rec["_value"], rec["_ms_per_step"], rec["_launches"], rec["_frozen"] = tokens / seconds, seconds * 1e3, int(launches), frozen_info
+
+    # ---- end to end through the public API with host buffers: H2D of the step's inputs, D2H of its result
+    if not args.no_e2e:
+        pin = lambda t: t.cpu().pin_memory()
+        hq, hkt, hvt, hlg = pin(q), pin(kt), pin(vt), pin(lgs[0])
+        h_old, h_new = pin(n_old), pin(n_new)
+        dq, dkt, dvt, dlg = torch.empty_like(q), torch.empty_like(kt), torch.empty_like(vt), lgs[0]
+        d_old, d_new = torch.empty(B, dtype=torch.int32, device=device), torch.empty(B, dtype=torch.int32, device=device)
+        h_acc = torch.empty(B, dtype=torch.int32).pin_memory()
+        h_out = torch.empty(B, cfg.max_depth + 1, dtype=torch.int32).pin_memory()
+        h_nn = torch.empty(B, dtype=torch.int32).pin_memory()
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hkt, hvt, hlg)) + 2 * B * 4
+        d2h = (h_acc.numel() + h_out.numel() + h_nn.numel()) * 4
+        s0 = 2 * (Wm + K) + K
+        ke = int(max(3, min(K, total - s0 - 2, 2000.0 / max(step_ms[full] + h2d / 20e6, 1e-3))))     # a couple of seconds of steps
+        e2e_tokens = 0.0
+        with torch.cuda.stream(stream):
+            def e2e_step(s):
+                r = s % R
+                dq.copy_(hq, non_blocking=True); dkt.copy_(hkt, non_blocking=True); dvt.copy_(hvt, non_blocking=True)
+                dlg.copy_(hlg, non_blocking=True)
+                d_old.copy_(h_old[s], non_blocking=True); d_new.copy_(h_new[s], non_blocking=True)
+                tr = trees[s]
+                if args.separate_calls:
+                    cb.cb_update(toks_d, d_old, d_new)
+                    cb.cb_draft_tree(toks_d, d_new, tr)
+                else:
+                    cb.cb_update_draft_tree(toks_d, d_old, d_new, tr)
+                at = ftree if full else tr
+                cb.cb_tree_attn(dq, kps[r], vps[r], bt_d, ctx_d, dkt, dvt, at["mask"], at["n_nodes"], out=out, max_ctx=max_ctx)
+                cb.cb_accept(at, logits=dlg, res=res)
+                h_acc.copy_(res["n_accept"], non_blocking=True); h_out.copy_(res["out_tokens"], non_blocking=True)
+                h_nn.copy_(at["n_nodes"], non_blocking=True)
+                stream.synchronize()
+                return float(h_nn.sum())                     # the tree nodes this step verified
+            for s in range(s0, s0 + 2):
+                e2e_step(s)
+            t0 = time.perf_counter()
+            for s in range(s0 + 2, s0 + 2 + ke):
+                e2e_tokens += e2e_step(s)
+            e2e_s = time.perf_counter() - t0
+        if world > 1:
+            e2e_s, e2e_tokens = reduce_over_ranks(e2e_s, e2e_tokens, device)
+        rec["_e2e"] = {"value": e2e_tokens / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                       "ms_per_step": 1e3 * e2e_s / ke, "steps": ke}
+        del hq, hkt, hvt, hlg, dq, dkt, dvt
     st, counters = cb.cb_poll_status()
     assert st == 0, "device status %d" % st
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-    hbm_peak, tf_peak, peak_kind = peaks()
-    nn_mean = nn_percall.mean(axis=0)                       # trees of the steps the per-call graphs ran
-    a_bytes = attn_bytes(cfg, ctx, nn_mean)
-    attn_ms = float(per_med[2])
-    t_mem, t_cmp = a_bytes / (hbm_peak * 1e9), attn_flops(cfg, ctx, nn_mean, float(np.sum(nn_mean * 4))) / (tf_peak * 1e12)
-    traffic = ATTN_TRAFFIC["bytes_per_launch"].get(cfg.name) if ATTN_TRAFFIC["sources_sha1"] == attn_sources_sha1() else None
-    if t_mem >= t_cmp:
-        roof = {"bound": "hbm", "achieved": a_bytes / (attn_ms * 1e-3) / 1e9, "peak": hbm_peak, "unit": "GB/s"}
-    else:
-        fl = attn_flops(cfg, ctx, nn_mean, float(np.sum(nn_mean * 4)))
-        roof = {"bound": "tensor", "achieved": fl / (attn_ms * 1e-3) / 1e12, "peak": tf_peak, "unit": "TFLOP/s"}
-    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": traffic, "kernel": "cb_tree_attn (attention kernel, plus its merge pass where the launch is not in cluster mode)",
-                 "ms_per_launch": attn_ms, "peak_source": peak_kind + " (MEASURED_PEAKS.json)" if peak_kind == "measured" else "fallback",
-                 "algorithmic_bytes": a_bytes})
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-        "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": cfg.name, "batch": B, "tree_cap": T, "mean_tree_nodes": float(nn_attn.mean()),
-                   "context": [int(ctx.min()), int(ctx.max())], "l2": "rotating %d copies of K/V pool and logits (%.0f MB)" %
-                   (R, R * (pool_bytes + logit_bytes) / 1e6), "launch": "CUDA graph of the timed steps, replayed %d times, median" % reps,
-                   "trees": "synthetic full" if args.full_trees else "drafted", "frozen_table": frozen_info,
-                   "calls": ("cb_update, cb_draft_tree" if args.separate_calls else "cb_update_draft_tree") + ", cb_tree_attn, cb_accept",
-                   "parallelism": "replicas x%d" % world},
-        "clocks": clocks, "gpu_launches": int(launches),
-        "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                "ms_per_step": 1e3 * e2e_s / K},
-        "roofline": roof,
-        "per_call_ms": {"cb_update": float(per_med[0]), "cb_draft_tree": float(per_med[1]), "cb_tree_attn": float(per_med[2]),
-                        "cb_accept": float(per_med[3]), "cb_update_draft_tree": float(per_med[4])},
-        "accept_gbs": (float(np.sum(nn_mean)) * cfg.vocab * 4) / (float(per_med[3]) * 1e-3) / 1e9,
-        "counters": counters,
-    }
-    if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(cfg, (ctx, toks, lens, bt), None)
-    print(json.dumps(line))
+    rec["_counters"] = counters
+    if world == 1 and rank == 0 and not args.no_cpu_baseline:
+        tokens_c, seconds_c, sample = oracle_sample(cfg, ctx, toks, lens, bt, 2, full)
+        rec["_cpu"] = {"value": tokens_c / seconds_c, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample}
+    return rec
+
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
     if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    head_name = args.config or HEADLINE
+    names = [args.config] if args.config else (FULL_SIZE if world == 1 else [HEADLINE])
+    per_config, head = [], None
+    for name in names:
+        rec = measure(args, name, rank, world, device, name == head_name)
+        torch.cuda.empty_cache()
+        if name == head_name:
+            head = rec
+        per_config.append({k: v for k, v in rec.items() if not k.startswith("_")})
+    if rank == 0:
+        full = not args.drafted_headline
+        line = {
+            "metric": METRIC, "value": head["_value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": head["_ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": head_name, "batch": head["batch"], "tree_cap": head["tree_cap"],
+                       "trees": "synthetic full (%d nodes each)" % head["tree_cap"] if full else "drafted",
+                       "value_drafted_trees": head["value_drafted_trees"], "ms_per_step_drafted_trees": head["ms_per_step_drafted_trees"],
+                       "mean_tree_nodes_drafted": head["mean_tree_nodes_drafted"], "context": head["context"], "l2": head["l2"],
+                       "launch": "CUDA graph of the timed steps, replayed %d times, median" % head["replays"],
+                       "frozen_table": head["_frozen"],
+                       "calls": ("cb_update, cb_draft_tree" if args.separate_calls else "cb_update_draft_tree") + ", cb_tree_attn, cb_accept",
+                       "parallelism": "replicas x%d" % world},
+            "clocks": head["clocks"], "gpu_launches": head["_launches"],
+            "roofline": head["roofline"], "per_call_ms": head["per_call_ms"], "accept": head["accept"],
+            "prompt_ingest": head["prompt_ingest"], "per_config": per_config, "counters": head["_counters"],
+        }
+        if "_e2e" in head:
+            line["e2e"] = head["_e2e"]
+        if "_cpu" in head:
+            line["cpu_baseline"] = head["_cpu"]
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
         dist.destroy_process_group()
+
+
+def rank_plumbing_only(rank, world):
+    """The rank start-up and result gathering alone, on CPU (gloo): what a test of the multi-rank launch can run without a GPU."""
+    import torch
+    import torch.distributed as dist
+    dist.init_process_group("gloo")
+    seconds, units = reduce_over_ranks(0.010 * (rank + 1), 1000.0 + rank, torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"n_gpus": world, "seconds": seconds, "units": units}))
+    dist.destroy_process_group()
 
 
 def main():
     args = parse()
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.rank_plumbing_only:
+        rank_plumbing_only(rank, world)
+        return
     if args.impl == "reference":
         run_reference(args, rank, world)
         return

@@ -54,12 +54,15 @@ __device__ void accept_walk(int b, int Dmax, const int32_t* tk, const int32_t* p
             good = good && (tk[c] == target_s[p]);
             c = p;
         }
-        if (good) best = max(best, ((uint32_t)de[i] << 8) | (uint32_t)(255 - i));
+        // a depth outside [0, Dmax] cannot come from the drafter (malformed input): such a node counts as unverified, so the
+        // winner's depth always fits the output rows
+        const int d = de[i];
+        if (good && d >= 0 && d <= Dmax) best = max(best, ((uint32_t)d << 8) | (uint32_t)(255 - i));
     }
     best = __reduce_max_sync(CB_FULL, best);
     int node = n > 0 ? 255 - (int)(best & 255u) : 0;
     int m = n > 0 ? (int)(best >> 8) : 0;
-    if (m > Dmax) m = Dmax;
+    if (node >= n) { node = 0; m = 0; }                        // nothing verified, not even the root (malformed input)
     for (int k = lane; k < Dmax; k += 32) accept_nodes[(size_t)b * Dmax + k] = -1;
     for (int k = lane; k <= Dmax; k += 32) out_tokens[(size_t)b * (Dmax + 1) + k] = -1;
     __syncwarp();
@@ -199,7 +202,7 @@ __global__ void __launch_bounds__(128) cb_accept_ids_kernel(int B, int T, int Dm
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int b = blockIdx.x * 4 + w;
     if (b >= B) return;
-    const int n = n_nodes[b];
+    const int n = min(max(n_nodes[b], 0), T);
     for (int k = lane; k < T; k += 32) {
         const int32_t tg = k < n ? target_in[(size_t)b * T + k] : -1;
         s_target[w][k] = tg;

@@ -43,3 +43,17 @@ def test_two_ranks_report_max_time_and_summed_units():
         p.join(timeout=120)
         assert p.exitcode == 0
     assert abs(seconds - 0.020) < 1e-12 and units == 2001.0
+
+
+def test_gpus_flag_starts_its_own_ranks():
+    """`bench.py --gpus 2` outside a torchrun launch starts two ranks itself; here with the CPU-only plumbing mode, so that
+    the start-up and the gathering run without a GPU."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rank-plumbing-only"], env=env,
+                       capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = [l for l in r.stdout.splitlines() if l.startswith("{")][-1]
+    d = json.loads(line)
+    assert d["n_gpus"] == 2 and abs(d["seconds"] - 0.020) < 1e-12 and d["units"] == 2001.0
