@@ -49,6 +49,7 @@ def parse(argv=None):
     ap.add_argument("--separate-calls", action="store_true", help="cb_update and cb_draft_tree as two launches")
     ap.add_argument("--frozen", type=int, default=0, metavar="TOKENS",
                     help="attach a frozen table built on the GPU from a synthetic corpus of this many tokens (0 = none)")
+    ap.add_argument("--flags", type=int, default=0, help="cb_config.flags for the context (4 = tree attention as pairs of CTAs)")
     ap.add_argument("--rank-plumbing-only", action="store_true", help=argparse.SUPPRESS)
     return ap.parse_args(argv)
 
@@ -315,7 +316,7 @@ def measure(args, cfg_name, rank, world, device, headline):
     out = torch.empty_like(q)
     max_ctx = int(ctx.max())
 
-    cb = Cacheback.from_config(cfg, device=device)
+    cb = Cacheback.from_config(cfg, device=device, flags=args.flags)
     prefill = np.minimum(ctx + 1, lens).astype(np.int32)
     total = 3 * (Wm + K) + 8
     assert int((lens - prefill).min()) > ADVANCE * total + T, "stream too short for this many steps"

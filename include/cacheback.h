@@ -54,7 +54,10 @@ enum { CB_DTYPE_F32 = 0, CB_DTYPE_BF16 = 1 };
 /* cb_config.flags */
 enum {
     CB_FLAG_NO_FOLLOWER_REFRESH = 1u, /* re-inserting a stored follower leaves its recency unchanged     */
-    CB_FLAG_ATTN_CUDA_CORES = 2u      /* run tree attention on the plain CUDA-core kernel (debug aid)    */
+    CB_FLAG_ATTN_CUDA_CORES = 2u,     /* run tree attention on the plain CUDA-core kernel (debug aid)    */
+    CB_FLAG_ATTN_CTA_PAIRS = 4u       /* tree attention of multi-row-tile launches (head_dim 128) as pairs of
+                                         CTAs issuing 2-CTA tensor-core products; measured slower than the
+                                         default on the configurations benchmarked, kept as an alternative */
 };
 
 /*
@@ -96,8 +99,8 @@ void cb_destroy(cb_ctx* ctx);
 cb_status cb_reset(cb_ctx* ctx, const int32_t* dev_seq_mask, void* stream);
 
 /*
- * Table update (Section 3.1 insertion rules; Section 3.2 "sliding window over the accepted tokens";
- * Section 3.3 prompt initialisation = the same call with n_old = 0).
+ * Table update (Section 3.1 insertion rules; Section 3.2, last paragraph: every leader-follower window that the newly
+ * accepted tokens complete is inserted; Section 3.3 prompt initialisation = the same call with n_old = 0).
  *   tokens   int32 [batch, row_stride]  token history of every sequence
  *   n_old    int32 [batch]  tokens already ingested by earlier calls
  *   n_new    int32 [batch]  tokens valid now (n_new >= n_old; n_new <= row_stride)
@@ -182,6 +185,10 @@ cb_status cb_tree_add_branches(cb_ctx* ctx, const int32_t* branches, const int32
  * Row (b, i, h) = softmax_j(scale * q.k_j) v_j over j in {cached tokens of kv head h / (Hq/Hkv)}
  * U {tree nodes in mask row i}; fp32 accumulation and softmax, output rounded to bf16.
  * All base pointers must be 16-byte aligned.
+ * Keys and values are fetched a tile at a time and what lies outside a row's key set is given probability 0, not skipped,
+ * so everything a tile covers must be finite (0 x NaN would reach the output): all T rows of k_tree / v_tree of every
+ * sequence, including rows >= n_nodes, and the slots of a sequence's last, partly filled page beyond ctx_len.  Pages past
+ * the last one are never read.  Buffers from an allocator that does not clear them must be zeroed once.
  */
 typedef struct {
     const void* q;
@@ -256,9 +263,9 @@ typedef struct {
 cb_status cb_kv_commit(cb_ctx* ctx, const cb_kv_commit_args* args, void* stream);
 
 /*
- * Frozen table (Section 3.3: besides the dynamic table, a second table is prepared offline from frequent
- * leader-follower pairs of a large corpus; a decoding step first queries the dynamic table to form the draft tree and
- * then the frozen one to grow the tree further while the size cap allows; the frozen table ignores insertions).
+ * Frozen table (Section 3.3): a second, read-only table built offline from the most frequent leader-follower pairs of a
+ * corpus.  A step drafts from the dynamic table first and then lets the frozen table add branches while the tree is below
+ * its size cap; insertions never reach it.
  *
  * A frozen table is one device buffer owned by the caller, of cb_frozen_bytes() bytes, 256-byte aligned, shared by every
  * sequence and every context that attaches it, and only read by the step calls.  LL and FL must equal the context's;

@@ -45,7 +45,7 @@ struct Table {
     uint64_t clock = 0;              // incremented by every insert and every query
     std::map<Key, Entry> leaders;
 
-    // Section 3.1, "The table updates its entries by accepting a leader-follower pair".
+    // Section 3.1, insertion rule: a (leader, follower) pair creates the leader with that follower, or appends / refreshes the follower.
     void insert(const int32_t* L, const int32_t* F) {
         clock++;
         Key lk(L, L + LL), fk(F, F + FL);

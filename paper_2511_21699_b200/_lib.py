@@ -8,7 +8,7 @@ SO_PATH = os.path.join(HERE, "libcacheback.so")
 
 CB_OK = 0
 CB_DTYPE_F32, CB_DTYPE_BF16 = 0, 1
-CB_FLAG_NO_FOLLOWER_REFRESH, CB_FLAG_ATTN_CUDA_CORES = 1, 2
+CB_FLAG_NO_FOLLOWER_REFRESH, CB_FLAG_ATTN_CUDA_CORES, CB_FLAG_ATTN_CTA_PAIRS = 1, 2, 4
 CB_ERR_STATIC_LIMIT = 7
 CB_ERR_KV_FULL = 8
 CB_STATIC_MAX_BATCH, CB_STATIC_MAX_ROWS = 1024, 8192

@@ -1,11 +1,15 @@
-// Tree attention: work decomposition shared by the tensor-core kernel and the merge pass.
+// Tree attention: work decomposition shared by the tensor-core kernels and the merge pass.
 //
 // Work is measured in key tiles of 128 keys.  Sequence b has tiles_b = ceil(ctx_b / 128) + 1 of them (the
 // last one holds the tree's own keys).  A unit is one (sequence, kv head, row group): a row group is a
 // pair of 128-row tiles (row = node_local * G + g, NPT = 128 / G nodes per tile), or a single tile when
-// the whole tree fits one tile; only row tiles that hold valid nodes form units.  All units, in
-// (sequence, kv head, row group) order, laid end to end give one global sequence of key tiles; it is cut
-// into `nc` equal ranges, one per persistent CTA (a stream-K split).  Starting a unit costs about as much as two or
+// the whole tree fits one tile; only row tiles that hold valid nodes form units.  All units laid end to end give one
+// global sequence of key tiles; it is cut into `nc` equal ranges, one per persistent CTA (or CTA pair): a stream-K split.
+// The order of the units is (row group, sequence, kv head), row group outermost: the units that stream the same keys and
+// values (one (sequence, kv head), all its row groups) then lie a fixed fraction of the whole sequence apart, so that they
+// are worked on at the same time by different CTAs and the keys and values are fetched from HBM once and found in L2 by
+// the others; with the row group innermost one CTA would stream them again and again, each time after everything else
+// it holds has passed through L2.  Starting a unit costs about as much as two or
 // three tiles (query load, pipeline refill, epilogue), so every unit is preceded by that many padding positions in the
 // sequence: they carry no work, they only make a CTA that handles many short units receive fewer tiles.  A CTA therefore finishes whole
 // units, plus at most one unit it shares with earlier CTAs and one it shares with later CTAs; shared
@@ -44,6 +48,8 @@ struct CbSeqShape {
     int n, ctx, tiles, mtn, RG;
     int ov;               // padding positions in front of each unit of this sequence
     long long W;          // positions (padding + key tiles) of all units of this sequence
+    // positions of this sequence's units of row group rg (all kv heads); 0 if the tree has no such row group
+    __device__ __forceinline__ long long w_of(int Hkv, int rg) const { return rg < RG ? (long long)Hkv * (tiles + ov) : 0ll; }
 };
 
 __device__ __forceinline__ CbSeqShape cb_seq_shape(const CbAttnParams& p, int b) {
@@ -62,8 +68,11 @@ __device__ __forceinline__ long long cb_range_start(long long total, int nc, int
 // CTA whose range holds global tile x.
 __device__ __forceinline__ int cb_cta_of(long long total, int nc, long long x) { return (int)(((x + 1) * nc - 1) / total); }
 
-// Warp-collective: total weight of all sequences, and the sequence holding global tile g (with the
-// global index at which that sequence starts).  Every lane gets the results.
+// Row groups a launch can have per sequence (trees of max_nodes nodes).
+__device__ __forceinline__ int cb_max_row_groups(const CbAttnParams& p) { return p.MT == 1 ? 1 : (p.MT + 1) / 2; }
+
+// Warp-collective: total weight of all sequences, and the (row group, sequence) holding global position g (with the
+// global index at which that sequence's units of that row group start).  Every lane gets the results.
 __device__ __forceinline__ long long cb_sched_total(const CbAttnParams& p, int lane) {
     long long tot = 0;
     for (int base = 0; base < p.B; base += 32) {
@@ -75,29 +84,33 @@ __device__ __forceinline__ long long cb_sched_total(const CbAttnParams& p, int l
     }
     return tot;
 }
-__device__ __forceinline__ void cb_sched_locate(const CbAttnParams& p, long long g, int lane, int* b_out, long long* pre_out) {
+__device__ __forceinline__ void cb_sched_locate(const CbAttnParams& p, long long g, int lane, int* rg_out, int* b_out, long long* pre_out) {
     long long run = 0;
-    int fb = p.B;
+    int frg = cb_max_row_groups(p), fb = p.B;
     long long fpre = 0;
-    for (int base = 0; base < p.B; base += 32) {
-        const int b = base + lane;
-        const long long w = b < p.B ? cb_seq_shape(p, b).W : 0;
-        long long inc = w;
+    for (int rg = 0; rg < cb_max_row_groups(p) && fb == p.B; ++rg) {
+        for (int base = 0; base < p.B; base += 32) {
+            const int b = base + lane;
+            const long long w = b < p.B ? cb_seq_shape(p, b).w_of(p.Hkv, rg) : 0;
+            long long inc = w;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const long long t = __shfl_up_sync(CB_FULL, inc, o);
-            if (lane >= o) inc += t;
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long t = __shfl_up_sync(CB_FULL, inc, o);
+                if (lane >= o) inc += t;
+            }
+            const long long pre = run + inc - w;
+            const uint32_t hit = __ballot_sync(CB_FULL, w > 0 && g >= pre && g < pre + w);
+            if (hit) {
+                const int l = __ffs(hit) - 1;
+                frg = rg;
+                fb = base + l;
+                fpre = __shfl_sync(CB_FULL, pre, l);
+                break;
+            }
+            run += __shfl_sync(CB_FULL, inc, 31);
         }
-        const long long pre = run + inc - w;
-        const uint32_t hit = __ballot_sync(CB_FULL, w > 0 && g >= pre && g < pre + w);
-        if (hit) {
-            const int l = __ffs(hit) - 1;
-            fb = base + l;
-            fpre = __shfl_sync(CB_FULL, pre, l);
-            break;
-        }
-        run += __shfl_sync(CB_FULL, inc, 31);
     }
+    *rg_out = frg;
     *b_out = fb;
     *pre_out = fpre;
 }
@@ -109,17 +122,18 @@ struct CbUnit {
 
 // Walks the units of the range [g, g1).  Every role of a CTA runs its own copy and sees the same units.
 struct CbWalker {
-    long long g, g1, pre;
-    int b;
+    long long g, g1, pre;     // pre: global position at which the units of (rg, b) start
+    int rg, b;
+    long long w;              // positions of the units of (rg, b)
     CbSeqShape s;
     bool fixed, fixed_left;   // cluster mode: the CTA has exactly one share of one unit (or none)
     CbUnit fu;
-    __device__ __forceinline__ void init(const CbAttnParams& p, long long g0, long long g1_, int b0, long long pre0) {
-        g = g0; g1 = g1_; b = b0; pre = pre0; fixed = false; fixed_left = false;
-        if (g < g1) s = cb_seq_shape(p, b);
+    __device__ __forceinline__ void init(const CbAttnParams& p, long long g0, long long g1_, int rg0, int b0, long long pre0) {
+        g = g0; g1 = g1_; rg = rg0; b = b0; pre = pre0; fixed = false; fixed_left = false; w = 0;
+        if (g < g1) { s = cb_seq_shape(p, b); w = s.w_of(p.Hkv, rg); }
     }
     __device__ __forceinline__ void init_fixed(const CbUnit& u0) {
-        g = 0; g1 = 0; b = 0; pre = 0; fixed = true; fixed_left = u0.t1 > u0.t0; fu = u0;
+        g = 0; g1 = 0; rg = 0; b = 0; pre = 0; w = 0; fixed = true; fixed_left = u0.t1 > u0.t0; fu = u0;
     }
     __device__ __forceinline__ bool next(const CbAttnParams& p, CbUnit* u) {
         if (fixed) {
@@ -130,18 +144,23 @@ struct CbWalker {
         }
         while (true) {
             if (g >= g1) return false;
-            while (g >= pre + s.W) { pre += s.W; ++b; s = cb_seq_shape(p, b); }
+            while (g >= pre + w) {                            // on to the next sequence that has this row group, then to the next row group
+                pre += w;
+                if (++b == p.B) { b = 0; ++rg; }
+                s = cb_seq_shape(p, b);
+                w = s.w_of(p.Hkv, rg);
+            }
             const long long off = g - pre;
             const int vt = s.tiles + s.ov;                    // positions of one unit
-            const int j = (int)(off / vt);
-            const int v0 = (int)(off - (long long)j * vt);
+            const int kh = (int)(off / vt);
+            const int v0 = (int)(off - (long long)kh * vt);
             const int v1 = (int)min((long long)vt, (long long)v0 + (g1 - g));
             g += v1 - v0;
             u->t0 = max(v0 - s.ov, 0);
             u->t1 = max(v1 - s.ov, 0);
             if (u->t1 <= u->t0) continue;                     // only padding of this unit falls into the range
-            u->b = b; u->kh = j / s.RG; u->rg = j % s.RG; u->tiles = s.tiles; u->n = s.n; u->ctx = s.ctx;
-            u->nrt = p.MT == 1 ? 1 : min(2, s.mtn - 2 * u->rg);
+            u->b = b; u->kh = kh; u->rg = rg; u->tiles = s.tiles; u->n = s.n; u->ctx = s.ctx;
+            u->nrt = p.MT == 1 ? 1 : min(2, s.mtn - 2 * rg);
             return true;
         }
     }

@@ -27,242 +27,9 @@
 
 #include <mutex>
 
-#include "cb_attn.cuh"
+#include "cb_tc_dev.cuh"
 
 namespace {
-
-constexpr long long kWaitCycles = 1ll << 32;     // bound of every wait, in SM clock cycles (about two seconds)
-constexpr uint32_t kSuspendNs = 20000;
-constexpr float kRowSumLimit = 1048576.f;        // a tile's row sum of P above which the row takes a new reference maximum
-constexpr int kThreads = 384;
-constexpr uint32_t kTmemCols = 512;
-
-struct TcMaps { CUtensorMap k_pool, v_pool, k_tree, v_tree, q; };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t n) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(n) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Potentially blocking test of a barrier phase: the hardware suspends the thread until the phase completes
-// or a time limit of about kSuspendNs passes, so waiting warps do not take issue slots from working ones.
-__device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
-    return ok;
-}
-// Bounded wait. Returns false when the wait ran out or another role already gave up; the first to run out
-// records CB_ERR_TIMEOUT and raises the CTA's abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
-    if (mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (true) {
-        if (mbar_try(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) break;
-    }
-    *abort_flag = 1;
-    atomicCAS(status, 0u, (uint32_t)CB_ERR_TIMEOUT);
-    return false;
-}
-
-// Cluster-scope helpers: address of a shared-memory location in another CTA of the cluster, arrival on a barrier there
-// (releasing this thread's earlier writes to the cluster), a 16-byte store there, and a bounded wait that acquires them.
-__device__ __forceinline__ uint32_t cluster_addr(uint32_t local, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t remote_bar) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
-}
-__device__ __forceinline__ void st_cluster_v4(uint32_t raddr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(raddr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_cluster(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
-    return ok;
-}
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* status) {
-    if (mbar_try_cluster(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (true) {
-        if (mbar_try_cluster(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) break;
-    }
-    *abort_flag = 1;
-    atomicCAS(status, 0u, (uint32_t)CB_ERR_TIMEOUT);
-    return false;
-}
-
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cta.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-
-// The cached context is read once per call: its copies are marked as the first to leave L2, so that what the other kernels
-// of a step keep coming back to (the n-gram tables) is still there after 100 MB of keys and values have passed through.
-__device__ __forceinline__ uint64_t l2_evict_first_policy() {
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ void tma_load_4d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3, uint64_t pol) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cta.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-#define CB_R32(a, o) "=r"(a[o + 0]), "=r"(a[o + 1]), "=r"(a[o + 2]), "=r"(a[o + 3]), "=r"(a[o + 4]), "=r"(a[o + 5]), \
-    "=r"(a[o + 6]), "=r"(a[o + 7]), "=r"(a[o + 8]), "=r"(a[o + 9]), "=r"(a[o + 10]), "=r"(a[o + 11]), "=r"(a[o + 12]), \
-    "=r"(a[o + 13]), "=r"(a[o + 14]), "=r"(a[o + 15]), "=r"(a[o + 16]), "=r"(a[o + 17]), "=r"(a[o + 18]), "=r"(a[o + 19]), \
-    "=r"(a[o + 20]), "=r"(a[o + 21]), "=r"(a[o + 22]), "=r"(a[o + 23]), "=r"(a[o + 24]), "=r"(a[o + 25]), "=r"(a[o + 26]), \
-    "=r"(a[o + 27]), "=r"(a[o + 28]), "=r"(a[o + 29]), "=r"(a[o + 30]), "=r"(a[o + 31])
-#define CB_W32(a, o) "r"(a[o + 0]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]), "r"(a[o + 5]), \
-    "r"(a[o + 6]), "r"(a[o + 7]), "r"(a[o + 8]), "r"(a[o + 9]), "r"(a[o + 10]), "r"(a[o + 11]), "r"(a[o + 12]), \
-    "r"(a[o + 13]), "r"(a[o + 14]), "r"(a[o + 15]), "r"(a[o + 16]), "r"(a[o + 17]), "r"(a[o + 18]), "r"(a[o + 19]), \
-    "r"(a[o + 20]), "r"(a[o + 21]), "r"(a[o + 22]), "r"(a[o + 23]), "r"(a[o + 24]), "r"(a[o + 25]), "r"(a[o + 26]), \
-    "r"(a[o + 27]), "r"(a[o + 28]), "r"(a[o + 29]), "r"(a[o + 30]), "r"(a[o + 31])
-
-// 32 consecutive 32-bit columns of this thread's TMEM lane -> registers a[o .. o+32)
-#define CB_TMEM_LD32(a, o, taddr)                                                                                    \
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, "   \
-                 "%13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, "  \
-                 "[%32];" : CB_R32(a, o) : "r"(taddr) : "memory")
-#define CB_TMEM_ST32(a, o, taddr)                                                                                    \
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, " \
-                 "%12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, "   \
-                 "%31};" ::CB_W32(a, o), "r"(taddr) : "memory")
-#define CB_RW32(a) "+r"(a[0]), "+r"(a[1]), "+r"(a[2]), "+r"(a[3]), "+r"(a[4]), "+r"(a[5]), "+r"(a[6]), "+r"(a[7]), "+r"(a[8]), \
-    "+r"(a[9]), "+r"(a[10]), "+r"(a[11]), "+r"(a[12]), "+r"(a[13]), "+r"(a[14]), "+r"(a[15]), "+r"(a[16]), "+r"(a[17]), "+r"(a[18]), \
-    "+r"(a[19]), "+r"(a[20]), "+r"(a[21]), "+r"(a[22]), "+r"(a[23]), "+r"(a[24]), "+r"(a[25]), "+r"(a[26]), "+r"(a[27]), "+r"(a[28]), \
-    "+r"(a[29]), "+r"(a[30]), "+r"(a[31])
-// Waits for this thread's outstanding TMEM loads; naming the destination registers keeps their uses below the wait.
-#define CB_TMEM_WAIT_LD32(a) asm volatile("tcgen05.wait::ld.sync.aligned;" : CB_RW32(a) :: "memory")
-#define CB_TMEM_ST16(a, o, taddr)                                                                                    \
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, " \
-                 "%12, %13, %14, %15};" ::"r"(a[o + 0]), "r"(a[o + 1]), "r"(a[o + 2]), "r"(a[o + 3]), "r"(a[o + 4]),  \
-                 "r"(a[o + 5]), "r"(a[o + 6]), "r"(a[o + 7]), "r"(a[o + 8]), "r"(a[o + 9]), "r"(a[o + 10]),           \
-                 "r"(a[o + 11]), "r"(a[o + 12]), "r"(a[o + 13]), "r"(a[o + 14]), "r"(a[o + 15]), "r"(taddr) : "memory")
-// 32-byte store: one instruction fills a whole DRAM sector of this thread's output row
-__device__ __forceinline__ void st_global_v8(void* ptr, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t a4, uint32_t a5, uint32_t a6,
-                                             uint32_t a7) {
-    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(ptr), "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(a4), "r"(a5), "r"(a6),
-                 "r"(a7) : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-// Two fp32 values in one 64-bit register pair, for the packed fp32x2 arithmetic of sm_100.
-__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
-__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
-// Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major or MN-major.
-__host__ __device__ constexpr uint32_t make_idesc(int M, int N, bool b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
-           ((uint32_t)(M >> 4) << 24);
-}
-
-// Low and high 32-bit words of a shared-memory matrix descriptor (128-byte swizzle, 1024-byte stride between
-// 8-row groups).  All operands live below 256 KB, so stepping the low word by (bytes >> 4) moves the start address.
-__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) { return ((saddr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16); }
-constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-
-// One MMA issuer thread feeds the tensor pipe, so the instructions between two MMAs are kept to a minimum: each
-// of the blocks below issues all MMAs of one 128 x 128 x D (or 128 x D x 128) product from a single asm statement.
-#define CB_MMA_SS_STEP(OFF)                                                                                          \
-    "add.u32 ra, %1, " #OFF ";\n\tadd.u32 rb, %2, " #OFF ";\n\tmov.b64 da, {ra, %3};\n\tmov.b64 db, {rb, %3};\n\t"  \
-    "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pt;\n\t"
-// S[tmem] = Q[smem, K-major] * K[smem, K-major]^T over D.  qlo / klo: low descriptor words of the first 16-wide slice.
-template <int D>
-__device__ __forceinline__ void mma_s_block(uint32_t d_tmem, uint32_t qlo, uint32_t klo, uint32_t idesc) {
-    if (D == 128) {
-        asm volatile(
-            "{\n\t.reg .pred pt, pf;\n\t.reg .b64 da, db;\n\t.reg .b32 ra, rb;\n\t"
-            "setp.eq.u32 pt, %4, %4;\n\tsetp.ne.u32 pf, %4, %4;\n\t"
-            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pf;\n\t"
-            CB_MMA_SS_STEP(2) CB_MMA_SS_STEP(4) CB_MMA_SS_STEP(6) CB_MMA_SS_STEP(1024) CB_MMA_SS_STEP(1026) CB_MMA_SS_STEP(1028)
-            CB_MMA_SS_STEP(1030) "}"
-            ::"r"(d_tmem), "r"(qlo), "r"(klo), "r"(kDescHi), "r"(idesc) : "memory");
-    } else {
-        asm volatile(
-            "{\n\t.reg .pred pt, pf;\n\t.reg .b64 da, db;\n\t.reg .b32 ra, rb;\n\t"
-            "setp.eq.u32 pt, %4, %4;\n\tsetp.ne.u32 pf, %4, %4;\n\t"
-            "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, pf;\n\t"
-            CB_MMA_SS_STEP(2) CB_MMA_SS_STEP(4) CB_MMA_SS_STEP(6) "}"
-            ::"r"(d_tmem), "r"(qlo), "r"(klo), "r"(kDescHi), "r"(idesc) : "memory");
-    }
-}
-#define CB_MMA_TS_STEP(K)                                                                                            \
-    "add.u32 ra, %1, 8 * " #K ";\n\tadd.u32 rb, %2, 128 * " #K ";\n\tmov.b64 db, {rb, %3};\n\t"                     \
-    "tcgen05.mma.cta_group::1.kind::f16 [%0], [ra], db, %4, pt;\n\t"
-// O[tmem] (+)= P[tmem, packed bf16] * V[smem, MN-major] over the tile's 128 keys.  vlo: low descriptor word of the V tile.
-__device__ __forceinline__ void mma_pv_block(uint32_t d_tmem, uint32_t p_tmem, uint32_t vlo, uint32_t idesc, uint32_t accum) {
-    asm volatile(
-        "{\n\t.reg .pred pt, pa;\n\t.reg .b64 db;\n\t.reg .b32 ra, rb;\n\t"
-        "setp.eq.u32 pt, %4, %4;\n\tsetp.ne.u32 pa, %5, 0;\n\t"
-        "mov.b64 db, {%2, %3};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, pa;\n\t"
-        CB_MMA_TS_STEP(1) CB_MMA_TS_STEP(2) CB_MMA_TS_STEP(3) CB_MMA_TS_STEP(4) CB_MMA_TS_STEP(5) CB_MMA_TS_STEP(6) CB_MMA_TS_STEP(7) "}"
-        ::"r"(d_tmem), "r"(p_tmem), "r"(vlo), "r"(kDescHi), "r"(idesc), "r"(accum) : "memory");
-}
-
-template <int REGS> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS)); }
-template <int REGS> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS)); }
-__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
-}
 
 template <int D>
 struct Cfg {
@@ -281,8 +48,14 @@ struct Cfg {
     static constexpr uint32_t O_COL = 256;                   // TMEM columns: S0 at 0, S1 at 128, O0 at 256, O1 at 256 + D
 };
 
-struct SchedSmem { long long g0, g1, pre0; int b0; int c_b, c_kh, c_t0, c_t1, c_tiles, c_n, c_ctx, c_has; };
+struct SchedSmem { long long g0, g1, pre0; int b0, rg0; int c_b, c_kh, c_t0, c_t1, c_tiles, c_n, c_ctx, c_has; };
 static_assert(sizeof(SchedSmem) <= 64, "the schedule block is followed by the tmem base and the abort flag");
+
+}  // namespace
+
+#include "cb_attn_pair.cuh"
+
+namespace {
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -344,23 +117,23 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             s_sched->c_has = sh.RG > 0 ? 1 : 0;
             s_sched->c_t0 = sh.RG > 0 ? (int)((long long)sh.tiles * rank / p.cs) : 0;
             s_sched->c_t1 = sh.RG > 0 ? (int)((long long)sh.tiles * (rank + 1) / p.cs) : 0;
-            s_sched->g0 = 0; s_sched->g1 = 0; s_sched->pre0 = 0; s_sched->b0 = 0;
+            s_sched->g0 = 0; s_sched->g1 = 0; s_sched->pre0 = 0; s_sched->b0 = 0; s_sched->rg0 = 0;
         }
     } else if (warp == 0) {
         // this CTA's range of the global tile sequence
         const long long tot = cb_sched_total(p, lane);
         const long long g0 = cb_range_start(tot, p.nc, cta), g1 = cb_range_start(tot, p.nc, cta + 1);
-        int b0 = 0;
+        int b0 = 0, rg0 = 0;
         long long pre0 = 0;
-        if (g0 < g1) cb_sched_locate(p, g0, lane, &b0, &pre0);
-        if (lane == 0) { s_sched->g0 = g0; s_sched->g1 = g1; s_sched->b0 = b0; s_sched->pre0 = pre0; }
+        if (g0 < g1) cb_sched_locate(p, g0, lane, &rg0, &b0, &pre0);
+        if (lane == 0) { s_sched->g0 = g0; s_sched->g1 = g1; s_sched->b0 = b0; s_sched->rg0 = rg0; s_sched->pre0 = pre0; }
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *s_tmem;
     const long long g0 = s_sched->g0, g1 = s_sched->g1, pre0 = s_sched->pre0;
-    const int b0 = s_sched->b0;
+    const int b0 = s_sched->b0, rg0 = s_sched->rg0;
     CbWalker wk;
     if (p.cs > 0) {
         // the peers' barriers must exist before anything arrives on them
@@ -371,7 +144,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
         u0.tiles = s_sched->c_tiles; u0.n = s_sched->c_n; u0.ctx = s_sched->c_ctx; u0.nrt = 1;
         wk.init_fixed(u0);
     } else {
-        wk.init(p, g0, g1, b0, pre0);
+        wk.init(p, g0, g1, rg0, b0, pre0);
     }
     CbUnit u;
 
@@ -933,14 +706,14 @@ __global__ void __launch_bounds__(256) cb_attn_merge_kernel(const CbAttnParams p
     const long long tot = cb_sched_total(p, lane);
     bool nothing = tot <= 0;
     long long g0 = 0, g1 = 0, pre = 0, ustart = 0;
-    int b = 0, j = 0, vt = 1;
+    int b = 0, rg = 0, j = 0, vt = 1;
     CbSeqShape s = {};
     if (!nothing) {
         g0 = cb_range_start(tot, p.nc, c); g1 = cb_range_start(tot, p.nc, c + 1);
         nothing = g1 <= g0 || g1 >= tot;                      // empty range, or the last range
     }
     if (!nothing) {
-        cb_sched_locate(p, g1 - 1, lane, &b, &pre);
+        cb_sched_locate(p, g1 - 1, lane, &rg, &b, &pre);
         s = cb_seq_shape(p, b);
         const long long off = g1 - 1 - pre;
         vt = s.tiles + s.ov;                                  // positions of one unit: padding, then its key tiles
@@ -956,7 +729,7 @@ __global__ void __launch_bounds__(256) cb_attn_merge_kernel(const CbAttnParams p
         return;
     }
     const int c_last = cb_cta_of(tot, p.nc, ustart + vt - 1);
-    const int kh = j / s.RG, rg = j % s.RG;
+    const int kh = j;                                         // units of (row group, sequence) are its kv heads
     const int nrt = p.MT == 1 ? 1 : min(2, s.mtn - 2 * rg);
     const int RT = p.NPT * p.G;
     constexpr int PER = D / 32;
@@ -1088,6 +861,56 @@ bool g_attr_set[2][kMaxDevices];
 ShapeMemo g_shape_memo[kShapeMemo];
 int g_shape_used = 0, g_shape_next = 0;
 
+int g_pairs[kMaxDevices];              // CTA pairs that can be resident at once (0 = not asked yet, -1 = none)
+
+// On request (CB_FLAG_ATTN_CTA_PAIRS), launches with two or more row tiles per unit and head_dim 128 run as pairs of CTAs
+// (cb_attn_pair.cuh): as many pairs as can be resident together, each taking an equal range of the global tile sequence.
+cb_status launch_pairs(CbAttnParams p, const TcMaps& maps, cudaStream_t st, int num_sms, int device, bool* done) {
+    *done = false;
+    const int di = device >= 0 && device < kMaxDevices ? device : -1;
+    if (di < 0) return CB_OK;
+    int npairs;
+    {
+        std::lock_guard<std::mutex> lock(g_launch_mutex);
+        if (g_pairs[di] == 0) {
+            g_pairs[di] = -1;
+            if (cudaFuncSetAttribute(cb_attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PairCfg::SMEM_ALLOC) == cudaSuccess) {
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3((unsigned)(num_sms / 2 * 2)); cfg.blockDim = dim3(kPairThreads); cfg.dynamicSmemBytes = PairCfg::SMEM_ALLOC;
+                cudaLaunchAttribute at[1];
+                at[0].id = cudaLaunchAttributeClusterDimension;
+                at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+                cfg.attrs = at; cfg.numAttrs = 1;
+                int n = 0;
+                if (cudaOccupancyMaxActiveClusters(&n, cb_attn_pair_kernel, &cfg) == cudaSuccess && n > 0) g_pairs[di] = n < num_sms / 2 ? n : num_sms / 2;
+            }
+            (void)cudaGetLastError();
+        }
+        npairs = g_pairs[di];
+    }
+    if (npairs <= 0) return CB_OK;
+    // The units that stream the same keys (the row groups of one (sequence, kv head)) lie 1 / row-groups of the tile sequence
+    // apart: with a number of ranges that is a multiple of the row groups they are at the same point of their ranges at the
+    // same time, so that one fetch from HBM serves all of them.
+    const int row_groups = (p.MT + 1) / 2;
+    if (npairs > row_groups) npairs -= npairs % row_groups;
+    p.nc = npairs; p.cs = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * npairs)); cfg.blockDim = dim3(kPairThreads); cfg.dynamicSmemBytes = PairCfg::SMEM_ALLOC; cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 2;
+    CB_CUDA(cudaLaunchKernelEx(&cfg, cb_attn_pair_kernel, p, maps));
+    CB_CUDA(cb_launch_pdl(cb_attn_merge_kernel<128>, dim3(p.nc, 4), dim3(256), 0, st, p));
+    cb_count_launch(2);
+    CB_CUDA(cudaGetLastError());
+    *done = true;
+    return CB_OK;
+}
+
 template <int D>
 cb_status launch(CbAttnParams p, const TcMaps& maps, cudaStream_t st, int num_sms, int device) {
     {
@@ -1154,6 +977,7 @@ std::mutex g_map_mutex;
 
 cb_status cb_attn_launch_tensor(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t st) {
     if (p.P != 16) return CB_ERR_UNSUPPORTED;
+    const bool pairs = p.D == 128 && p.MT > 1 && (ctx->cfg.flags & CB_FLAG_ATTN_CTA_PAIRS);
     const MapKey key = {p.q, p.k_pool, p.v_pool, p.k_tree, p.v_tree, p.D, p.Hq, p.Hkv, p.P, p.T, p.B, p.G, p.NPT, p.num_pages};
     TcMaps maps;
     bool hit = false;
@@ -1172,6 +996,11 @@ cb_status cb_attn_launch_tensor(cb_ctx* ctx, const CbAttnParams& p, cudaStream_t
         const int slot = g_map_used < kMapCache ? g_map_used++ : (g_map_next++ % kMapCache);
         g_map_keys[slot] = key;
         g_map_vals[slot] = maps;
+    }
+    if (pairs) {
+        bool done = false;
+        const cb_status r = launch_pairs(p, maps, st, ctx->num_sms, ctx->device, &done);
+        if (r != CB_OK || done) return r;
     }
     return p.D == 128 ? launch<128>(p, maps, st, ctx->num_sms, ctx->device) : launch<64>(p, maps, st, ctx->num_sms, ctx->device);
 }

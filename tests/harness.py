@@ -137,28 +137,33 @@ def oracle_attn_rows_by_head(oracle, cfg, prob, mask, rows, threads=None):
 
 
 def shared_unit_rows(cfg, ctx, n, n_ctas, seed=11):
-    """One (b, h, i) row in every unit of tree attention that two persistent CTAs share.
+    """One (b, h, i) row in every unit of tree attention that two persistent CTAs (or CTA pairs) share.
 
     Restates the decomposition the attention kernel documents: work is counted in 128-key tiles; sequence b has
     ceil(ctx_b / 128) + 1 of them (the last holds the tree's own keys); a row tile packs 128 / G nodes with the G query
     heads of a kv head; a unit is one (sequence, kv head, row group), a row group being a pair of row tiles (one when the
     whole tree cap fits one); every unit is preceded by 3 padding positions when its sequence has two or more row tiles,
-    else 2; all units laid end to end in (sequence, kv head, row group) order are cut into n_ctas equal ranges,
-    range c = [total * c // n_ctas, total * (c + 1) // n_ctas)."""
+    else 2; all units laid end to end in (row group, sequence, kv head) order, row group outermost, are cut into n_ctas
+    equal ranges, range c = [total * c // n_ctas, total * (c + 1) // n_ctas)."""
     G, Hkv, T = cfg.gqa, cfg.n_kv_heads, cfg.max_nodes
     npt = 128 // G
     MT = -(-T // npt)
     rng = np.random.default_rng(seed)
-    units = []                                             # (first position, padding, tiles, b, kh, rg, row tiles)
-    pos = 0
+    shapes = []
     for b in range(cfg.batch):
         nb = int(min(max(n[b], 0), T))
         tiles = -(-int(ctx[b]) // 128) + 1
         mtn = -(-nb // npt)
         RG = (1 if mtn > 0 else 0) if MT == 1 else (mtn + 1) // 2
-        ov = 3 if mtn >= 2 else 2
-        for kh in range(Hkv):
-            for rg in range(RG):
+        shapes.append((tiles, mtn, RG, 3 if mtn >= 2 else 2))
+    units = []                                             # (first position, padding, tiles, b, kh, rg, row tiles)
+    pos = 0
+    for rg in range(1 if MT == 1 else (MT + 1) // 2):
+        for b in range(cfg.batch):
+            tiles, mtn, RG, ov = shapes[b]
+            if rg >= RG:
+                continue
+            for kh in range(Hkv):
                 nrt = 1 if MT == 1 else min(2, mtn - 2 * rg)
                 units.append((pos, ov, tiles, b, kh, rg, nrt))
                 pos += ov + tiles

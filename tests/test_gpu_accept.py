@@ -72,7 +72,7 @@ def test_accept_logits_small(oracle, name, full, dtype):
     assert r["n_accept"].max() >= 1                      # planted matches are found
 
 
-@pytest.mark.parametrize("name,dtype", [("c3_8b_gqa", "f32"), ("c3_8b_gqa", "bf16"), ("c5_70b_long", "bf16")])
+@pytest.mark.parametrize("name,dtype", [("c3_8b_gqa", "f32"), ("c3_8b_gqa", "bf16"), ("c5_70b_long", "bf16"), ("c5_70b_long", "f32")])
 def test_accept_logits_full_size_sampled(oracle, name, dtype):
     cfg = W.get_config(name)
     _run(cfg, dtype, False, [0, 1, cfg.batch // 2, cfg.batch - 1], oracle)

@@ -123,6 +123,10 @@ def _times16(bits):
 
 @pytest.mark.parametrize("cfg,ctxs", [(CLUSTER_4, [600]), (SMALL_GQA, [300, 300, 300, 257, 140])])
 def test_attn_score_jumps_between_and_inside_tiles(oracle, cfg, ctxs):
+    _jumps(oracle, cfg, ctxs)
+
+
+def _jumps(oracle, cfg, ctxs, flags=0):
     """Keys of the second key tile, and of the first tile past its first 40 keys, are 16 times larger: their scores lie
     dozens of powers of two above the reference maximum the softmax has in use when it meets them (taken from an
     earlier tile, or from the first 32 scores of a share's first tile), so the one-pass form must give way to the
@@ -141,7 +145,7 @@ def test_attn_score_jumps_between_and_inside_tiles(oracle, cfg, ctxs):
             kp[pg, t % P] = _times16(kp[pg, t % P])
     d = device_attn_inputs(cfg, prob)
     d["k_pool"] = torch.from_numpy(kp.view(np.int16)).cuda().view(torch.bfloat16)
-    cb = Cacheback.from_config(cfg)
+    cb = Cacheback.from_config(cfg, flags=flags)
     lse = torch.zeros((B, cfg.n_q_heads, T), dtype=torch.float32, device="cuda")
     out = torch.empty((B, T, cfg.n_q_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda")
     cb.cb_tree_attn(d["q"], d["k_pool"], d["v_pool"], d["block_table"], d["ctx_len"], d["k_tree"], d["v_tree"],
@@ -202,3 +206,17 @@ def test_attn_long_units_mixed_row_tiles_repeated(oracle):
         hh = torch.tensor([r[0] for r in rows], device="cuda")
         ii = torch.tensor([r[1] for r in rows], device="cuda")
         _check_rows(bf16_to_f64(out[b, ii, hh]), lse[b, hh, ii].cpu().numpy().astype(np.float64), ref, ref_lse, (cfg.name, b))
+
+
+@pytest.mark.parametrize("case", ["ragged", "c3", "jumps"])
+def test_attn_cta_pair_kernel(oracle, case):
+    """The alternative kernel for launches with several row tiles per (sequence, kv head): pairs of CTAs issuing 2-CTA
+    tensor-core products, each CTA holding half of every K and V tile.  Ragged and empty contexts, the 8B-shaped batch at
+    full size, and scores that jump far above the running reference."""
+    from paper_2511_21699_b200 import _lib
+    if case == "ragged":
+        _run(SMALL_GQA, oracle, False, _all, flags=_lib.CB_FLAG_ATTN_CTA_PAIRS, ctx_override=[0, 1, 16, 256, 299])
+    elif case == "c3":
+        _run(W.get_config("c3_8b_gqa"), oracle, True, _sampled(3, 3, 6), flags=_lib.CB_FLAG_ATTN_CTA_PAIRS)
+    else:
+        _jumps(oracle, SMALL_GQA, [300, 300, 300, 257, 140], flags=_lib.CB_FLAG_ATTN_CTA_PAIRS)

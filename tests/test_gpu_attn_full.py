@@ -45,7 +45,7 @@ def test_attn_full_size_whole_sequences_random_rows_and_seams(oracle, name):
                     dev(mask.view(np.int32)), dev(n), out=out, lse=lse, max_ctx=int(prob.ctx.max()))
     torch.cuda.synchronize()
     assert cb.cb_poll_status()[0] == 0
-    n_ctas = min(torch.cuda.get_device_properties(0).multi_processor_count, 160)
+    n_ctas = min(torch.cuda.get_device_properties(0).multi_processor_count, 160)   # ranges of the stream-K split: one per SM
     whole, rand, seams = _rows(cfg, prob, n, n_ctas)
     assert len(whole) == 2 * cfg.n_q_heads * T and len(rand) >= 4096 and len(seams) >= n_ctas // 2, (len(whole), len(rand), len(seams))
     rows = np.array(whole + rand + seams, np.int64)

@@ -181,11 +181,10 @@ def test_shared_unit_rows_lie_in_units_cut_by_a_range_boundary():
     # brute force: label every position of the global sequence with its unit and whether it is a key tile
     G, npt = cfg.gqa, 128 // cfg.gqa
     label = []
-    for b in range(cfg.batch):
+    for b in range(cfg.batch):                             # 64 nodes x 4 heads = two row tiles = one row group
         tiles = -(-int(ctx[b]) // 128) + 1
         for kh in range(cfg.n_kv_heads):
-            for rg in range(1):                            # 64 nodes x 4 heads = two row tiles = one row group
-                label += [(b, kh, False)] * 3 + [(b, kh, True)] * tiles
+            label += [(b, kh, False)] * 3 + [(b, kh, True)] * tiles
     total = len(label)
     cut_units = set()
     for c in range(1, 148):
@@ -194,3 +193,22 @@ def test_shared_unit_rows_lie_in_units_cut_by_a_range_boundary():
             cut_units.add(label[g][:2])
     assert {(b, h // G) for b, h, i in rows} == cut_units
     assert all(0 <= i < cfg.max_nodes for _, _, i in rows)
+    # several row groups (128 nodes x 8 heads = 8 row tiles = 4 row groups): the row group is the outermost index
+    cfg = W.get_config("c5_70b_long")
+    ctx = W.ctx_lens(cfg)
+    n = np.full(cfg.batch, cfg.max_nodes, np.int32)
+    rows = shared_unit_rows(cfg, ctx, n, 74)
+    label = []
+    for rg in range(4):
+        for b in range(cfg.batch):
+            tiles = -(-int(ctx[b]) // 128) + 1
+            for kh in range(cfg.n_kv_heads):
+                label += [(b, kh, rg, False)] * 3 + [(b, kh, rg, True)] * tiles
+    total = len(label)
+    cut_units = set()
+    for c in range(1, 74):
+        g = total * c // 74
+        if label[g - 1][:3] == label[g][:3] and label[g - 1][3] and label[g][3]:
+            cut_units.add(label[g][:3])
+    npt = 128 // cfg.gqa
+    assert {(b, h // cfg.gqa, i // (2 * npt)) for b, h, i in rows} == cut_units
