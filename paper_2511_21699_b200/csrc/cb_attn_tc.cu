@@ -385,15 +385,19 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     // visibility of the tile's 128 keys for this row: context keys below ctx, tree keys by the ancestor bits
                     const bool is_tree = i == nct;
                     const int kv = is_tree ? u.n : min(CB_KT, u.ctx - i * CB_KT);
-                    uint32_t vm[4];
+                    uint32_t vm[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+                    // A context tile that lies wholly inside the context needs no masks.  Rows that do not exist take the fast
+                    // path too: whatever they compute stays in their own row.
+                    bool all_vis = !is_tree && kv == CB_KT;
+                    if (!all_vis) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const int lo = kv - 32 * k;
-                        const uint32_t below = lo >= 32 ? 0xFFFFFFFFu : (lo <= 0 ? 0u : ((1u << lo) - 1u));
-                        vm[k] = row_valid ? (is_tree ? (mrow[k] & below) : below) : 0u;
+                        for (int k = 0; k < 4; ++k) {
+                            const int lo = kv - 32 * k;
+                            const uint32_t below = lo >= 32 ? 0xFFFFFFFFu : (lo <= 0 ? 0u : ((1u << lo) - 1u));
+                            vm[k] = row_valid ? (is_tree ? (mrow[k] & below) : below) : 0u;
+                        }
+                        all_vis = __all_sync(CB_FULL, !row_valid || (vm[0] & vm[1] & vm[2] & vm[3]) == 0xFFFFFFFFu);
                     }
-                    // rows that do not exist take the fast path too: whatever they compute stays in their own row
-                    const bool all_vis = __all_sync(CB_FULL, !row_valid || (vm[0] & vm[1] & vm[2] & vm[3]) == 0xFFFFFFFFu);
                     uint32_t sa[32], sb[32];
                     // Single pass, tried first on every tile: P against the reference maximum in use, held back in registers so
                     // that S is still whole if the tile has to be done again.  No row maximum is taken.  The reference exists
@@ -454,7 +458,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                         f2_unpack(lsa, l0, l1);
                         f2_unpack(lsb, l2, l3);
                         const float lt = (l0 + l1) + (l2 + l3);
-                        if (!__any_sync(CB_FULL, !(lt <= kRowSumLimit))) {
+                        if (!__any_sync(CB_FULL, row_valid && !(lt <= kRowSumLimit))) {   // rows that do not exist hold anything: they never ask
                             CB_TMEM_ST16(pk, 0, ts);
                             CB_TMEM_ST16(pk, 16, ts + 16);
                             CB_TMEM_ST16(pk, 32, ts + 32);
