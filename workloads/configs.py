@@ -66,5 +66,9 @@ CONFIGS["p_tuned"] = replace(CONFIGS["c2_7b"], name="p_tuned", LL=1, FL=3, LC=1 
 CONFIGS["p_fc40_evict"] = replace(CONFIGS["p_tuned"], name="p_fc40_evict", LC=512, FC=40)
 
 
+# The 70B shape on a batch small enough for a profiler capture (keys and values of 8 sequences: 1.1 GB).
+CONFIGS["c5_70b_b8"] = replace(CONFIGS["c5_70b_long"], name="c5_70b_b8", batch=8)
+
+
 def get_config(name: str) -> CbConfig:
     return CONFIGS[name]
