@@ -45,6 +45,7 @@ def parse(argv=None):
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-closed-loop", action="store_true")
     ap.add_argument("--drafted-headline", action="store_true", help="headline value from the drafter's own trees instead of full ones")
     ap.add_argument("--separate-calls", action="store_true", help="cb_update and cb_draft_tree as two launches")
     ap.add_argument("--frozen", type=int, default=0, metavar="TOKENS",
@@ -278,6 +279,98 @@ def run_reference(args, rank, world):
 
 
 # --------------------------------------------------------------------------------------------------------
+def closed_loop(args, cfg, ctx, toks, lens, tensors, device, frozen):
+    """The decoding loop with the token stream as the target model, wholly on the device: every step is cb_update_draft_tree
+    -> cb_tree_attn -> (target ids: the stream's continuation along matching paths) -> cb_accept -> cb_kv_commit, and the
+    sequences advance by what was accepted plus the bonus token.  32 steps in one CUDA graph.  Returns mean accepted tokens
+    per step (bonus token included), whether every emitted token equals the stream (speculative decoding is lossless), and
+    the step time."""
+    import torch
+    import workloads as W
+    from workloads import device as wdev
+    from workloads.tensors import TID
+    from paper_2511_21699_b200 import Cacheback
+    q, kt, vt, toks_d, out = tensors
+    B, T, Dm = cfg.batch, cfg.max_nodes, cfg.max_depth
+    KC = 32
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
+    margin = 4 * KC * (Dm + 1) + 16                         # room for the cache to grow (up to four replays of the graph)
+    prefill = np.minimum(ctx + 1, lens).astype(np.int32)
+    assert int((lens - prefill).min()) > KC * (Dm + 1) + Dm + 2, "stream too short for the closed loop"
+    from dataclasses import replace
+    bt, num_pages = W.make_block_table(replace(cfg, ctx_range=(cfg.ctx_range[0], cfg.ctx_range[1] + margin)), ctx + margin)
+    pshape = (num_pages, cfg.page_size, cfg.n_kv_heads, cfg.head_dim)
+    kp = wdev.fill_normal(torch.empty(pshape, dtype=torch.bfloat16, device=device), cfg.seed + 5, TID.K_POOL)
+    vp = wdev.fill_normal(torch.empty(pshape, dtype=torch.bfloat16, device=device), cfg.seed + 5, TID.V_POOL)
+    bt_d, ctx0, pre_d, zeros_d = dev(bt), dev(ctx), dev(prefill), dev(np.zeros(B, np.int32))
+    cb = Cacheback.from_config(cfg, device=device, flags=args.flags)
+    if frozen is not None:
+        cb.cb_frozen_attach(frozen)
+    tree, res = cb.alloc_tree(), cb.alloc_accept()
+    i32 = dict(dtype=torch.int32, device=device)
+    tgt = torch.empty(B, T, **i32)
+    pos_old, pos, ctx_d = torch.empty(B, **i32), torch.empty(B, **i32), torch.empty(B, **i32)
+    log_acc, log_tok, log_n = torch.zeros(KC, B, **i32), torch.zeros(KC, B, Dm + 1, **i32), torch.zeros(KC, B, **i32)
+    max_ctx = int(ctx.max()) + margin
+
+    def reset():
+        cb.cb_reset()
+        cb.cb_update_bulk(toks_d, zeros_d, pre_d)          # prompt initialisation
+        pos_old.copy_(pre_d); pos.copy_(pre_d); ctx_d.copy_(ctx0)
+
+    def step(s):
+        cb.cb_update_draft_tree(toks_d, pos_old, pos, tree)
+        cb.cb_tree_attn(q, kp, vp, bt_d, ctx_d, kt, vt, tree["mask"], tree["n_nodes"], out=out, max_ctx=max_ctx)
+        wdev.stream_targets(toks_d, pos, tree, cfg.vocab, tgt)
+        cb.cb_accept(tree, target_ids=tgt, res=res)
+        cb.cb_kv_commit(kp, vp, bt_d, ctx_d, kt, vt, res["n_accept"], res["accept_nodes"])
+        log_acc[s].copy_(res["n_accept"]); log_tok[s].copy_(res["out_tokens"]); log_n[s].copy_(tree["n_nodes"])
+        pos_old.copy_(pos)
+        pos.add_(res["n_accept"]).add_(1)
+
+    stream = torch.cuda.Stream(device=device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        reset()
+        step(0)                                             # eager, so that every kernel is loaded before the capture
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for s in range(KC):
+                step(s)
+        room = int((lens - prefill).min()) - Dm - 2
+        replays = int(max(1, min(4, room // (KC * (Dm + 1)))))   # the loop goes on from where the last replay left it
+        reset()
+        g.replay()                                          # warms the graph up
+        reset()
+        stream.synchronize()
+        ms, accs, toks_out, nns = 0.0, [], [], []
+        for rep_ in range(replays):
+            e0.record(stream)
+            g.replay()
+            e1.record(stream)
+            stream.synchronize()
+            ms += e0.elapsed_time(e1)
+            accs.append(log_acc.cpu().numpy()); toks_out.append(log_tok.cpu().numpy()); nns.append(log_n.cpu().numpy())
+    st, _ = cb.cb_poll_status()
+    assert st == 0, "device status %d in the closed loop" % st
+    acc, tok, nn = np.concatenate(accs), np.concatenate(toks_out), np.concatenate(nns)
+    steps = KC * replays
+    lossless = True
+    for b in range(B):
+        p0 = int(prefill[b])
+        emitted = np.concatenate([tok[s, b, :acc[s, b] + 1] for s in range(steps)])
+        lossless = lossless and bool(np.array_equal(emitted, toks[b, p0:p0 + len(emitted)]))
+    steps_tokens = float((acc + 1).sum())
+    return {"steps": steps, "steps_per_graph": KC, "ms_per_step": ms / steps, "mat": steps_tokens / (steps * B), "lossless": lossless,
+            "mat_definition": "tokens emitted per step and sequence: accepted draft tokens plus the bonus token",
+            "mean_tree_nodes": float(nn.mean()), "tree_tokens_per_s": float(nn.sum()) / (ms * 1e-3),
+            "emitted_tokens_per_s": steps_tokens / (ms * 1e-3),
+            "calls": "cb_update_draft_tree, cb_tree_attn, stream targets (workloads), cb_accept (ids), cb_kv_commit; positions advance on the device",
+            "paper_mat_context": {"no_frozen": 1.96, "dual": 2.42, "source": "Table 1, Vicuna 7B on SpecBench, 1x RTX 4090 (context only: other model, other data)"},
+            "frozen_table": frozen is not None}
+
+
 def measure(args, cfg_name, rank, world, device, headline):
     """Everything measured on one configuration.  Returns the record; a headline record also carries the pieces of the
     top-level line (keys that start with an underscore: whole-job value, end-to-end figure, launch count)."""
@@ -356,7 +449,7 @@ def measure(args, cfg_name, rank, world, device, headline):
             "bytes_per_window": entry_bytes + (cfg.FL + 2) * 4, "gbs": bulk_bytes / bulk_t / 1e9,
             "frac_of_hbm": bulk_bytes / bulk_t / 1e9 / pk["hbm_gbs"]}
 
-    frozen_info = None
+    frozen_info, ft = None, None
     if args.frozen > 0:
         # Stand-in for the paper's corpus sample: streams of the workload's own token distribution under other seeds.
         from paper_2511_21699_b200 import FrozenTable
@@ -505,9 +598,17 @@ def measure(args, cfg_name, rank, world, device, headline):
         rec["latency_bound"] = ("at batch 1 cb_update, cb_draft_tree and cb_accept move a few KB to a few MB per call through chains "
                                 "of dependent memory round trips: their time is launch plus round trips, not bandwidth")
 
+    def run_closed_loop():
+        if args.no_closed_loop or world > 1:
+            return
+        kps.clear(); vps.clear(); lgs.clear()              # the loop brings its own pool (with room to grow)
+        torch.cuda.empty_cache()
+        rec["closed_loop"] = closed_loop(args, cfg, ctx, toks, lens, (q, kt, vt, toks_d, out), device, ft)
+
     if not headline:
         st, counters = cb.cb_poll_status()
         assert st == 0, "device status %d" % st
+        run_closed_loop()
         return rec
 
     # ---- whole-job figures over ranks
@@ -565,6 +666,9 @@ def measure(args, cfg_name, rank, world, device, headline):
     st, counters = cb.cb_poll_status()
     assert st == 0, "device status %d" % st
     rec["_counters"] = counters
+    if not args.no_e2e:
+        del dlg
+    run_closed_loop()
     if world == 1 and rank == 0 and not args.no_cpu_baseline:
         tokens_c, seconds_c, sample = oracle_sample(cfg, ctx, toks, lens, bt, 2, full)
         rec["_cpu"] = {"value": tokens_c / seconds_c, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample}
@@ -603,7 +707,8 @@ def run_ours(args, rank, world, local_rank):
                        "parallelism": "replicas x%d" % world},
             "clocks": head["clocks"], "gpu_launches": head["_launches"],
             "roofline": head["roofline"], "per_call_ms": head["per_call_ms"], "accept": head["accept"],
-            "prompt_ingest": head["prompt_ingest"], "per_config": per_config, "counters": head["_counters"],
+            "prompt_ingest": head["prompt_ingest"], "closed_loop": head.get("closed_loop"), "per_config": per_config,
+            "counters": head["_counters"],
         }
         if "_e2e" in head:
             line["e2e"] = head["_e2e"]

@@ -29,6 +29,9 @@ def _load():
         _lib = C.CDLL(build())
         _lib.wl_fill_normal.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, C.c_float, C.c_int, C.c_void_p]
         _lib.wl_fill_normal.restype = C.c_int
+        _lib.wl_stream_targets.argtypes = [C.c_void_p, C.c_longlong, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                           C.c_int32, C.c_void_p, C.c_void_p]
+        _lib.wl_stream_targets.restype = C.c_int
     return _lib
 
 
@@ -44,3 +47,16 @@ def fill_normal(t: torch.Tensor, seed: int, tid: int):
 
 def normal_tensor(shape, dtype, seed, tid, device="cuda:0"):
     return fill_normal(torch.empty(shape, dtype=dtype, device=device), seed, tid)
+
+
+def stream_targets(tokens: torch.Tensor, seq_len: torch.Tensor, tree: dict, junk_base: int, out: torch.Tensor):
+    """Closed-loop stand-in for the target model (input generation): out[b, i] = the token of the stream `tokens[b]` that follows
+    node i's path if that path equals the stream's continuation after position seq_len[b] - 1 (the tree's root), else
+    junk_base + i.  All int32 CUDA tensors; tree = dict(tokens, parent, depth, n_nodes) as cb_draft_tree writes it."""
+    B, T = tree["tokens"].shape
+    rc = _load().wl_stream_targets(tokens.data_ptr(), tokens.stride(0), seq_len.data_ptr(), tree["tokens"].data_ptr(), tree["parent"].data_ptr(),
+                                   tree["depth"].data_ptr(), tree["n_nodes"].data_ptr(), B, T, junk_base, out.data_ptr(),
+                                   torch.cuda.current_stream().cuda_stream)
+    if rc != 0:
+        raise RuntimeError("wl_stream_targets failed with CUDA error %d" % rc)
+    return out

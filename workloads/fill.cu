@@ -33,3 +33,33 @@ extern "C" int wl_fill_normal(void* out, uint64_t n, uint64_t key, float scale, 
     else wl_fill_f32_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((float*)out, n, key, scale);
     return (int)cudaGetLastError();
 }
+
+// Closed-loop stand-in for the target model: the token stream itself.  target[b, i] = the stream token that follows node i's
+// path if the tokens on the path from the root to node i equal the stream's continuation (the root is the sequence's last
+// token), else a token outside the vocabulary range of the stream (so it never matches).  Input generation only: this is
+// what an LM head plus arg-max would hand to acceptance.
+__global__ void wl_stream_targets_kernel(const int32_t* tokens, long long row_stride, const int32_t* seq_len, const int32_t* tree_tok,
+                                         const int32_t* tree_par, const int32_t* tree_dep, const int32_t* n_nodes, int B, int T, int32_t junk_base,
+                                         int32_t* target) {
+    const int b = blockIdx.x, i = threadIdx.x;
+    if (b >= B || i >= T) return;
+    const int n = n_nodes[b], pos = seq_len[b];
+    int32_t out = -1;
+    if (i < n) {
+        const int32_t* s = tokens + (long long)b * row_stride;
+        bool on = true;
+        int c = i;
+        for (int guard = 0; guard < T && c > 0; ++guard) {
+            on = on && tree_tok[(long long)b * T + c] == s[pos - 1 + tree_dep[(long long)b * T + c]];
+            c = tree_par[(long long)b * T + c];
+        }
+        out = on ? s[pos + tree_dep[(long long)b * T + i]] : junk_base + i;
+    }
+    target[(long long)b * T + i] = out;
+}
+extern "C" int wl_stream_targets(const int32_t* tokens, long long row_stride, const int32_t* seq_len, const int32_t* tree_tok, const int32_t* tree_par,
+                                 const int32_t* tree_dep, const int32_t* n_nodes, int B, int T, int32_t junk_base, int32_t* target, void* stream) {
+    if (B <= 0 || T <= 0 || T > 1024) return 1;
+    wl_stream_targets_kernel<<<B, T, 0, (cudaStream_t)stream>>>(tokens, row_stride, seq_len, tree_tok, tree_par, tree_dep, n_nodes, B, T, junk_base, target);
+    return (int)cudaGetLastError();
+}
