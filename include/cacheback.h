@@ -46,7 +46,8 @@ typedef enum {
     CB_ERR_TIMEOUT = 5,     /* device: a bounded wait (mbarrier / flag) ran out                        */
     CB_ERR_UNSUPPORTED = 6,
     CB_ERR_STATIC_LIMIT = 7, /* cb_accept_static: the problem does not fit the built-in scratch array       */
-    CB_ERR_KV_FULL = 8       /* device: cb_kv_commit found a sequence whose pages cannot hold the new tokens   */
+    CB_ERR_KV_FULL = 8,      /* device: cb_kv_commit found a sequence whose pages cannot hold the new tokens   */
+    CB_ERR_CANARY = 9        /* checking build only: a guard word beside a workspace region was overwritten    */
 } cb_status;
 
 enum { CB_DTYPE_F32 = 0, CB_DTYPE_BF16 = 1 };
@@ -372,6 +373,15 @@ enum {
     CB_NUM_COUNTERS = 8
 };
 cb_status cb_poll_status(cb_ctx* ctx, cb_status* device_status, uint64_t* counters);
+
+/*
+ * 1 if this library is the checking build (compiled with -DCB_DEBUG), else 0.  No counterpart in the paper: the checking
+ * build is the stand-in for a memory checker.  In it every table slot, entry id, page id and node index that a kernel takes
+ * from memory is range-checked before use (a value out of range records CB_ERR_INVALID_ARG in the device status and the
+ * access is skipped; nothing traps), and every workspace region is followed by 256 guard bytes that cb_poll_status verifies
+ * (CB_ERR_CANARY if one changed).  cb_workspace_bytes is larger in that build.  Results are identical to the regular build.
+ */
+int cb_debug_build(void);
 
 /* Kernels launched by this library since the process started (host-side count). */
 uint64_t cb_launch_count(void);

@@ -4,13 +4,17 @@ import ctypes as C
 import os
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-SO_PATH = os.path.join(HERE, "libcacheback.so")
+# CACHEBACK_LIBRARY names another build of the library to load, e.g. the checking build libcacheback_debug.so.
+SO_PATH = os.environ.get("CACHEBACK_LIBRARY") or os.path.join(HERE, "libcacheback.so")
+SO_DEBUG_PATH = os.path.join(HERE, "libcacheback_debug.so")
 
 CB_OK = 0
 CB_DTYPE_F32, CB_DTYPE_BF16 = 0, 1
 CB_FLAG_NO_FOLLOWER_REFRESH, CB_FLAG_ATTN_CUDA_CORES, CB_FLAG_ATTN_CTA_PAIRS = 1, 2, 4
 CB_ERR_STATIC_LIMIT = 7
 CB_ERR_KV_FULL = 8
+CB_ERR_INVALID_ARG, CB_ERR_CANARY = 1, 9
+CB_GUARD_BYTES = 256
 CB_STATIC_MAX_BATCH, CB_STATIC_MAX_ROWS = 1024, 8192
 CB_NUM_COUNTERS = 8
 COUNTER_NAMES = ["inserts", "leader_evictions", "follower_evictions", "queries", "query_hits", "max_probe", "frozen_queries",
@@ -19,7 +23,7 @@ COUNTER_NAMES = ["inserts", "leader_evictions", "follower_evictions", "queries",
 EXPORTS = ["cb_workspace_bytes", "cb_create", "cb_destroy", "cb_reset", "cb_update", "cb_draft_tree", "cb_update_draft_tree",
            "cb_tree_attn", "cb_accept", "cb_table_dump", "cb_table_load", "cb_poll_status", "cb_launch_count",
            "cb_status_str", "cb_accept_static", "cb_kv_commit", "cb_frozen_bytes", "cb_frozen_load", "cb_frozen_dump",
-           "cb_frozen_attach", "cb_frozen_build_bytes", "cb_frozen_build", "cb_tree_add_branches", "cb_update_bulk"]
+           "cb_frozen_attach", "cb_frozen_build_bytes", "cb_frozen_build", "cb_tree_add_branches", "cb_update_bulk", "cb_debug_build"]
 
 
 class CbConfigC(C.Structure):
@@ -81,6 +85,7 @@ def load():
     L.cb_launch_count.argtypes = []
     L.cb_status_str.restype = C.c_char_p
     L.cb_status_str.argtypes = [i32]
+    L.cb_debug_build.argtypes = []
     for name in EXPORTS:
         if name not in ("cb_destroy", "cb_launch_count", "cb_status_str"):
             getattr(L, name).restype = i32

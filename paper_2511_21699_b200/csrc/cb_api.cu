@@ -33,18 +33,26 @@ cb_status cb_compute_layout(const cb_config* c, CbLayout* L) {
     L->nslots = ns;
     L->E = (uint32_t)align_up((size_t)c->LL + (size_t)c->FC * (1 + c->FL), 4);
     size_t B = (size_t)c->batch, o = 0;
-    L->off_hdr = o;      o = align_up(o + B * 4 * 4, 256);
-    L->off_index = o;    o = align_up(o + B * ns * 4, 256);
-    L->off_lstamp = o;   o = align_up(o + B * (size_t)c->LC * 4, 256);
-    L->off_entries = o;  o = align_up(o + B * (size_t)c->LC * L->E * 4, 256);
-    L->off_status = o;   o = align_up(o + 4 * 4, 256);
-    L->off_counters = o; o = align_up(o + CB_NUM_COUNTERS * 8, 256);
-    L->off_rowmax = o;   o = align_up(o + B * (size_t)c->max_nodes * 8, 256);
-    L->off_ticket = o;   o = align_up(o + B * 4, 256);
-    L->off_bulk_plan = o; o = align_up(o + B * 16, 256);
+    L->n_guards = 0;
+    // a region of `bytes` at the current offset; the checking build puts a guard area behind it
+    auto region = [&](size_t bytes) {
+        const size_t at = o;
+        o = align_up(o + bytes, 256);
+        if (CB_DEBUG_BUILD) { L->guard_off[L->n_guards++] = o; o += CB_GUARD_BYTES; }
+        return at;
+    };
+    L->off_hdr = region(B * 4 * 4);
+    L->off_index = region(B * ns * 4);
+    L->off_lstamp = region(B * (size_t)c->LC * 4);
+    L->off_entries = region(B * (size_t)c->LC * L->E * 4);
+    L->off_status = region(4 * 4);
+    L->off_counters = region(CB_NUM_COUNTERS * 8);
+    L->off_rowmax = region(B * (size_t)c->max_nodes * 8);
+    L->off_ticket = region(B * 4);
+    L->off_bulk_plan = region(B * 16);
     L->attn_max_units = CB_ATTN_MAX_UNITS;
     L->attn_part_floats = (size_t)L->attn_max_units * 128 * ((size_t)c->head_dim + 4);
-    L->off_attn_part = o; o = align_up(o + L->attn_part_floats * 4, 256);
+    L->off_attn_part = region(L->attn_part_floats * 4);
     L->total = o;
     return CB_OK;
 }
@@ -83,6 +91,7 @@ extern "C" cb_status cb_create(const cb_config* cfg, void* dev_workspace, size_t
     t.nslots = L.nslots; t.E = L.E;
     t.LL = cfg->LL; t.FL = cfg->FL; t.LC = cfg->LC; t.FC = cfg->FC;
     t.refresh = (cfg->flags & CB_FLAG_NO_FOLLOWER_REFRESH) ? 0u : 1u;
+    t.dbg_status = (uint32_t*)(c->ws + L.off_status);
     c->d_status = (uint32_t*)(c->ws + L.off_status);
     c->d_counters = (unsigned long long*)(c->ws + L.off_counters);
     c->d_rowmax = (unsigned long long*)(c->ws + L.off_rowmax);
@@ -91,16 +100,21 @@ extern "C" cb_status cb_create(const cb_config* cfg, void* dev_workspace, size_t
     c->d_attn_part = (float*)(c->ws + L.off_attn_part);
     c->attn_part_floats = L.attn_part_floats;
     c->attn_max_units = L.attn_max_units;
+    c->n_guards = L.n_guards;
+    for (int g = 0; g < L.n_guards; ++g) c->guard_off[g] = L.guard_off[g];
     // Empty tables: header and index zero; entries and stamps need no initialisation (count = 0).
     bool ok = cudaMemset(c->ws + L.off_hdr, 0, L.off_lstamp - L.off_hdr) == cudaSuccess &&
-              cudaMemset(c->ws + L.off_status, 0, L.off_attn_part - L.off_status) == cudaSuccess &&
-              cudaDeviceSynchronize() == cudaSuccess;
+              cudaMemset(c->ws + L.off_status, 0, L.off_attn_part - L.off_status) == cudaSuccess;
+    for (int g = 0; g < L.n_guards && ok; ++g) ok = cudaMemset(c->ws + L.guard_off[g], CB_GUARD_BYTE, CB_GUARD_BYTES) == cudaSuccess;
+    ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) { delete c; return CB_ERR_CUDA; }
     *out = c;
     return CB_OK;
 }
 
 extern "C" void cb_destroy(cb_ctx* ctx) { delete ctx; }
+
+extern "C" int cb_debug_build(void) { return CB_DEBUG_BUILD; }
 
 __global__ void cb_reset_kernel(CbTables t, const int32_t* __restrict__ mask) {
     const int b = blockIdx.y;
@@ -202,6 +216,13 @@ extern "C" cb_status cb_poll_status(cb_ctx* ctx, cb_status* device_status, uint6
     CB_CUDA(cudaDeviceSynchronize());
     uint32_t st[4];
     CB_CUDA(cudaMemcpy(st, ctx->d_status, sizeof(st), cudaMemcpyDeviceToHost));
+    // checking build: the guard areas behind the workspace regions must still hold their fill
+    for (int g = 0; g < ctx->n_guards && st[0] == 0; ++g) {
+        unsigned char guard[CB_GUARD_BYTES];
+        CB_CUDA(cudaMemcpy(guard, ctx->ws + ctx->guard_off[g], CB_GUARD_BYTES, cudaMemcpyDeviceToHost));
+        for (int k = 0; k < CB_GUARD_BYTES; ++k)
+            if (guard[k] != CB_GUARD_BYTE) { st[0] = (uint32_t)CB_ERR_CANARY; break; }
+    }
     if (device_status) *device_status = (cb_status)st[0];
     if (st[0] != 0) CB_CUDA(cudaMemset(ctx->d_status, 0, sizeof(st)));
     if (counters) CB_CUDA(cudaMemcpy(counters, ctx->d_counters, CB_NUM_COUNTERS * 8, cudaMemcpyDeviceToHost));
@@ -219,6 +240,7 @@ extern "C" const char* cb_status_str(cb_status s) {
         case CB_ERR_UNSUPPORTED: return "unsupported device or shape";
         case CB_ERR_STATIC_LIMIT: return "problem larger than the built-in static scratch (see cb_accept_static)";
         case CB_ERR_KV_FULL: return "a sequence's pages cannot hold the committed tokens";
+        case CB_ERR_CANARY: return "a guard area beside a workspace region was overwritten (checking build)";
     }
     return "unknown status";
 }

@@ -212,7 +212,10 @@ cb_attn_pair_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                 int page = p.num_pages;                          // out of range: the copy fills zeros
                 if (active && i < nct) {
                     const int pidx = i * (CB_KT / 16) + pg_in_tile;
-                    if (pidx < npages) page = bt[pidx];
+                    if (pidx < npages) {
+                        page = bt[pidx];
+                        if (!cb_dbg_in(page, p.num_pages, p.status)) page = p.num_pages;   // the copy then fills zeros
+                    }
                 }
                 const uint32_t slot = c % C::NSLOT;
                 if (c >= (uint32_t)C::NSLOT && !(ok = mbar_wait(bar_free(slot), (c / C::NSLOT - 1) & 1, s_abort, p.status))) break;

@@ -23,7 +23,26 @@
 //                     else (tag << 20) | entry id, tag in [1, 4094] taken from the key's hash
 //   lstamp[LC]        leader recency stamps (dense, so the LRU scan reads 4 bytes per leader)
 //   entries[LC][E]    key[LL], follower stamps[FC] (0 = free), follower tokens[FC][FL]; E padded to 4 words
+// Checking build (-DCB_DEBUG): indices taken from memory are range-checked before use.  cb_dbg_in returns whether
+// 0 <= i < n; if not it records CB_ERR_INVALID_ARG in the device status and the caller skips the access.  In the regular
+// build it is a constant true and costs nothing.
+#ifdef CB_DEBUG
+#define CB_DEBUG_BUILD 1
+__device__ __forceinline__ bool cb_dbg_in(long long i, long long n, uint32_t* status) {
+    if (i >= 0 && i < n) return true;
+    if (status) atomicCAS(status, 0u, (uint32_t)CB_ERR_INVALID_ARG);
+    return false;
+}
+#else
+#define CB_DEBUG_BUILD 0
+__device__ __forceinline__ bool cb_dbg_in(long long, long long, uint32_t*) { return true; }
+#endif
+#define CB_GUARD_BYTES 256      // guard area behind every workspace region of the checking build
+#define CB_GUARD_BYTE 0xC5
+#define CB_MAX_GUARDS 12
+
 struct CbTables {
+    uint32_t* dbg_status;   // device status word for the checking build's range checks (may be null)
     uint32_t* hdr;
     uint32_t* index;
     uint32_t* lstamp;
@@ -76,6 +95,8 @@ struct cb_ctx {
     unsigned long long* d_rowmax;    // [batch * max_nodes] packed (value, index) maxima, zero between calls
     uint32_t* d_ticket;     // [batch] CTAs-finished counters, zero between calls
     uint32_t* d_bulk_plan;  // [batch][4] per-sequence plan of cb_update_bulk
+    size_t guard_off[CB_MAX_GUARDS];
+    int n_guards;
     float* d_attn_part;     // partial outputs of units shared between CTAs
     size_t attn_part_floats;
     int attn_max_units;     // partial row tiles available
@@ -87,6 +108,8 @@ struct CbLayout {
     size_t off_hdr, off_index, off_lstamp, off_entries, off_status, off_counters, off_rowmax, off_ticket, off_bulk_plan,
         off_attn_part, attn_part_floats, total;
     int attn_max_units;
+    size_t guard_off[CB_MAX_GUARDS];   // checking build: start of the guard area behind each region
+    int n_guards;
 };
 
 cb_status cb_compute_layout(const cb_config* cfg, CbLayout* L);

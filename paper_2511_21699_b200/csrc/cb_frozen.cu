@@ -33,6 +33,7 @@ CbTables cb_frozen_view(const cb_frozen_config* c, const CbFrozenLayout& L, void
     t.nslots = L.nslots; t.E = L.E;
     t.LL = c->LL; t.FL = c->FL; t.LC = c->LC; t.FC = c->FC;
     t.refresh = 0u;
+    t.dbg_status = nullptr;
     return t;
 }
 

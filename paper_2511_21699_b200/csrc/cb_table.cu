@@ -41,6 +41,7 @@ __device__ __forceinline__ Probe tbl_find(const CbTables& t, const CbSeq& s, int
             const int l = __ffs(cand) - 1;
             cand &= cand - 1;
             const uint32_t eid = __shfl_sync(CB_FULL, w, l) & CB_EID_MASK;
+            if (!cb_dbg_in(eid, t.LC, t.dbg_status)) continue;                // an index word naming an entry that cannot exist
             bool eq = true;
             if (FETCH == 2) {
                 const uint32_t* e = s.entries + (size_t)eid * t.E;
