@@ -4,6 +4,8 @@
 // index bucket with one coalesced load, compare the FC followers of an entry in parallel, and scan the
 // dense stamp array for the least recently used leader.  Recency is a per-sequence operation counter
 // ("clock"); a leader or follower stamp is the clock value of the operation that last touched it.
+#include <algorithm>
+
 #include "cb_common.cuh"
 
 namespace {
@@ -289,9 +291,10 @@ __global__ void cb_bulk_plan_kernel(CbTables t, int B, const int32_t* __restrict
     plan[b] = p;
 }
 
-// One insertion of the parallel path: c is the operation's stamp; no leader is ever evicted here.
-__device__ void tbl_insert_shared(const CbTables& t, const CbSeq& s, int32_t mykey, int32_t myfol, uint32_t c, int lane,
-                                  uint32_t* status, TblCounters& cnt) {
+// One insertion of the parallel path: c is the operation's stamp; no leader is ever evicted here.  Returns the leader's
+// entry id (-1 if the insertion failed).
+__device__ int tbl_insert_shared(const CbTables& t, const CbSeq& s, int32_t mykey, int32_t myfol, uint32_t c, int lane,
+                                 uint32_t* status, TblCounters& cnt) {
     cnt.inserts++;
     const uint64_t h = warp_hash(t, mykey);
     const uint32_t tagword = cb_hash_tag(h) << CB_EID_BITS;
@@ -304,7 +307,7 @@ __device__ void tbl_insert_shared(const CbTables& t, const CbSeq& s, int32_t myk
             if (lane == 0) s.lstamp[pr.eid] = c;
             tbl_put_follower(t, e, myfol, c, lane, cnt);
             __syncwarp();
-            return;
+            return pr.eid;
         }
         if (pr.eid != -1 || pr.free_slot == 0xFFFFFFFFu) break;
         if (eid < 0) {
@@ -325,21 +328,34 @@ __device__ void tbl_insert_shared(const CbTables& t, const CbSeq& s, int32_t myk
         uint32_t old = 0;
         if (lane == 0) old = atomicCAS(&s.index[pr.free_slot], CB_IDX_EMPTY, tagword | (uint32_t)eid);
         old = __shfl_sync(CB_FULL, old, 0);
-        if (old == CB_IDX_EMPTY) return;
+        if (old == CB_IDX_EMPTY) return eid;
         if (old == CB_IDX_TOMB) {                              // a deleted slot is as good as an empty one
             if (lane == 0) old = atomicCAS(&s.index[pr.free_slot], CB_IDX_TOMB, tagword | (uint32_t)eid);
             old = __shfl_sync(CB_FULL, old, 0);
-            if (old == CB_IDX_TOMB) return;
+            if (old == CB_IDX_TOMB) return eid;
         }
     }
     if (lane == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_PROBE_LIMIT);
+    return -1;
 }
 
-__global__ void __launch_bounds__(256) cb_update_bulk_kernel(CbTables t, int B, int WPS, const int32_t* __restrict__ tokens, int64_t row_stride,
+// The warp that owns a frequent leader meets it again and again (with unigram leaders a handful of tokens own a third of
+// the windows), and every insertion into a leader that is in the table is a chain of four dependent memory round trips.  So
+// every warp keeps the entries it touched last in shared memory (WAYS of them: key, follower stamps and tokens, leader
+// stamp): an insertion into a kept entry is the same follower-list code running on the shared-memory copy, and the copy goes
+// back to the table when its place is needed or the run ends.  No other warp touches these leaders during the run.
+__global__ void __launch_bounds__(256) cb_update_bulk_kernel(CbTables t, int B, int WPS, int WAYS, const int32_t* __restrict__ tokens, int64_t row_stride,
                                                              const int32_t* __restrict__ n_old, const int32_t* __restrict__ n_new,
                                                              const BulkPlan* __restrict__ plan, uint32_t* status, unsigned long long* counters) {
     CB_PDL_ENTRY();
+    extern __shared__ uint32_t bulk_smem[];
     const int lane = threadIdx.x & 31;
+    // this warp's kept entries: WAYS x (E words of the entry, then entry id + 1 (0 = free), leader stamp, last use, unused)
+    const uint32_t way_words = t.E + 4;
+    uint32_t* ways = bulk_smem + (size_t)(threadIdx.x >> 5) * WAYS * way_words;
+    for (int w = lane; w < WAYS; w += 32) ways[(size_t)w * way_words + t.E] = 0u;
+    __syncwarp();
+    uint32_t use_clock = 0;
     const int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int b = gw / WPS, wi = gw % WPS;
     if (b >= B) return;
@@ -376,8 +392,50 @@ __global__ void __launch_bounds__(256) cb_update_bulk_kernel(CbTables t, int B, 
                 const int i = (int)(pl.first + k0 + l);
                 const int32_t mykey = lane < t.LL ? row[i + lane] : 0;
                 const int32_t myfol = lane < t.FL ? row[i + t.LL + lane] : 0;
-                tbl_insert_shared(t, s, mykey, myfol, pl.clock0 + k0 + (uint32_t)l + 1u, lane, status, cnt);
+                const uint32_t c = pl.clock0 + k0 + (uint32_t)l + 1u;
+                // is the leader among the kept entries?  lane w compares way w's key
+                bool match = lane < WAYS && ways[(size_t)lane * way_words + t.E] != 0u;
+                for (int j = 0; j < t.LL; ++j) {
+                    const int32_t kj = __shfl_sync(CB_FULL, mykey, j);
+                    if (match) match = (int32_t)ways[(size_t)lane * way_words + j] == kj;
+                }
+                const uint32_t hit = __ballot_sync(CB_FULL, match);
+                ++use_clock;
+                if (hit) {
+                    uint32_t* e = ways + (size_t)(__ffs(hit) - 1) * way_words;
+                    cnt.inserts++;
+                    if (lane == 0) { e[t.E + 1] = c; e[t.E + 2] = use_clock; }
+                    tbl_put_follower(t, e, myfol, c, lane, cnt);
+                    __syncwarp();
+                    continue;
+                }
+                const int eid = tbl_insert_shared(t, s, mykey, myfol, c, lane, status, cnt);
+                if (eid < 0) continue;
+                // keep it: in a free way, else in place of the way used longest ago (whose copy goes back to the table first)
+                uint32_t u = lane < WAYS ? (ways[(size_t)lane * way_words + t.E] == 0u ? 0u : ways[(size_t)lane * way_words + t.E + 2]) : 0xFFFFFFFFu;
+                const uint32_t umin = __reduce_min_sync(CB_FULL, u);
+                uint32_t* e = ways + (size_t)(__ffs(__ballot_sync(CB_FULL, u == umin)) - 1) * way_words;
+                const uint32_t old = e[t.E];
+                if (old != 0u) {
+                    uint32_t* g = s.entries + (size_t)(old - 1u) * t.E;
+                    for (uint32_t k = lane; k < t.E; k += 32) g[k] = e[k];
+                    if (lane == 0) s.lstamp[old - 1u] = e[t.E + 1];
+                }
+                __syncwarp();
+                const uint32_t* g = s.entries + (size_t)eid * t.E;
+                for (uint32_t k = lane; k < t.E; k += 32) e[k] = __ldcg(g + k);
+                if (lane == 0) { e[t.E] = (uint32_t)eid + 1u; e[t.E + 1] = c; e[t.E + 2] = use_clock; }
+                __syncwarp();
             }
+        }
+        // the kept entries go back to the table
+        for (int w = 0; w < WAYS; ++w) {
+            const uint32_t* e = ways + (size_t)w * way_words;
+            const uint32_t id = e[t.E];
+            if (id == 0u) continue;
+            uint32_t* g = s.entries + (size_t)(id - 1u) * t.E;
+            for (uint32_t k = lane; k < t.E; k += 32) g[k] = e[k];
+            if (lane == 0) s.lstamp[id - 1u] = e[t.E + 1];
         }
     }
     if (lane == 0) {
@@ -661,12 +719,25 @@ extern "C" cb_status cb_update_bulk(cb_ctx* ctx, const int32_t* tokens, int64_t 
     const int B = ctx->cfg.batch;
     // enough warps per sequence to fill the GPU at small batch, fewer at large batch
     int wps = 1;
-    while (wps < 64 && (long long)B * wps * 2 <= (long long)ctx->num_sms * 16) wps *= 2;
+    while (wps < 256 && (long long)B * wps * 2 <= (long long)ctx->num_sms * 64) wps *= 2;
     BulkPlan* plan = reinterpret_cast<BulkPlan*>(ctx->d_bulk_plan);
     CB_CUDA(cb_launch_pdl(cb_bulk_plan_kernel, dim3((B + 127) / 128), dim3(128), 0, (cudaStream_t)stream, ctx->tables, B, n_old, n_new, plan));
     const long long warps = (long long)B * wps;
-    CB_CUDA(cb_launch_pdl(cb_update_bulk_kernel, dim3((unsigned)((warps + 7) / 8)), dim3(256), 0, (cudaStream_t)stream, ctx->tables, B, wps, tokens,
-                          row_stride, n_old, n_new, (const BulkPlan*)plan, ctx->d_status, ctx->d_counters));
+    // kept entries per warp: four, fewer where 96 KB of shared memory per CTA (8 warps) do not hold that many
+    const size_t way_bytes = ((size_t)ctx->tables.E + 4) * 4;
+    const int n_ways = (int)std::max<size_t>(1, std::min<size_t>(4, (96 * 1024) / (8 * way_bytes)));
+    const size_t smem = 8 * (size_t)n_ways * way_bytes;
+    if (smem > 200 * 1024) return CB_ERR_UNSUPPORTED;
+    if (smem > 48 * 1024) {
+        static size_t opted[64] = {0};                         // largest size opted into so far, per device
+        const int d = ctx->device & 63;
+        if (opted[d] < smem) {
+            CB_CUDA(cudaFuncSetAttribute(cb_update_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            opted[d] = smem;
+        }
+    }
+    CB_CUDA(cb_launch_pdl(cb_update_bulk_kernel, dim3((unsigned)((warps + 7) / 8)), dim3(256), smem, (cudaStream_t)stream, ctx->tables, B, wps, n_ways,
+                          tokens, row_stride, n_old, n_new, (const BulkPlan*)plan, ctx->d_status, ctx->d_counters));
     cb_count_launch(2);
     return CB_OK;
 }
