@@ -3,7 +3,8 @@
 //   nvcc -gencode arch=compute_100a,code=sm_100a -O3 -o mma_issue mma_issue.cu && ./mma_issue
 //
 // Throughput of tcgen05.mma blocks as the attention kernels issue them: time to issue n MMAs (128x128x16 per SM, bf16) and
-// time until their commit completes, for cta_group::1 and for a pair of CTAs with cta_group::2.  Operands are whatever
+// time until their commit completes, for cta_group::1 and for a pair of CTAs with cta_group::2; also 128xNx16 with N = 64
+// and N = 256 (cta_group::1, both operands from shared memory).  Operands are whatever
 // shared memory holds (zeroed); only timing matters.
 #include <cstdio>
 #include <cstdint>
@@ -36,7 +37,7 @@ __device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a_tmem, uint32_t blo
 }
 
 // res[0..]: per repetition (issue cycles, cycles until the commit's barrier completed)
-template <int CG, int TS>
+template <int CG, int TS, int NN = 128>
 __global__ void __launch_bounds__(128, 1) k(long long* res, int n_mma, int reps) {
     extern __shared__ __align__(1024) uint8_t smem[];
     __shared__ __align__(8) unsigned long long bar;
@@ -45,7 +46,7 @@ __global__ void __launch_bounds__(128, 1) k(long long* res, int n_mma, int reps)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint32_t rank = 0;
     if (CG == 2) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
-    for (int i = threadIdx.x; i < 64 * 1024 / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem + (sbase - smem_u32(smem)))[i] = 0u;
+    for (int i = threadIdx.x; i < (NN > 128 ? 112 : 64) * 1024 / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem + (sbase - smem_u32(smem)))[i] = 0u;
     if (warp == 0) {
         if (CG == 1) {
             asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&s_tmem)) : "memory");
@@ -66,7 +67,7 @@ __global__ void __launch_bounds__(128, 1) k(long long* res, int n_mma, int reps)
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = s_tmem;
     if (warp == 1 && lane == 0 && rank == 0) {
-        const uint32_t idesc = TS ? make_idesc(128 * CG, 128, true) : make_idesc(128 * CG, 128, false);
+        const uint32_t idesc = TS ? make_idesc(128 * CG, NN, true) : make_idesc(128 * CG, NN, false);
         const uint32_t alo = desc_lo(sbase, 16), blo = desc_lo(sbase + 32768, TS ? 16384 : 16);
         const uint32_t b = smem_u32(&bar);
         for (int r = 0; r < reps; ++r) {
@@ -97,17 +98,17 @@ __global__ void __launch_bounds__(128, 1) k(long long* res, int n_mma, int reps)
     }
 }
 
-template <int CG, int TS>
+template <int CG, int TS, int NN = 128>
 int run(long long* res, const char* name) {
-    const int smem = 64 * 1024 + 1024 + 1024;
-    CHK(cudaFuncSetAttribute(k<CG, TS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    const int smem = (NN > 128 ? 112 : 64) * 1024 + 1024 + 1024;   // B of N = 256: two 32 KB blocks from offset 32 KB and 48 KB
+    CHK(cudaFuncSetAttribute(k<CG, TS, NN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     for (int n : {1, 8, 16, 64}) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(CG); cfg.blockDim = dim3(128); cfg.dynamicSmemBytes = smem;
         cudaLaunchAttribute at[1];
         at[0].id = cudaLaunchAttributeClusterDimension; at[0].val.clusterDim.x = CG; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 1;
-        CHK(cudaLaunchKernelEx(&cfg, k<CG, TS>, res, n, 4));
+        CHK(cudaLaunchKernelEx(&cfg, k<CG, TS, NN>, res, n, 4));
         CHK(cudaDeviceSynchronize());
         long long h[12]; CHK(cudaMemcpy(h, res, sizeof(h), cudaMemcpyDeviceToHost));
         printf("%-28s n=%2d  issue %lld  commit %lld  until complete %lld cycles  (last of 4 repetitions; %.1f cycles per MMA)\n", name, n, h[9], h[10], h[11],
@@ -120,6 +121,8 @@ int main() {
     long long* res; CHK(cudaMalloc(&res, 64 * 8));
     if (run<1, 0>(res, "cta_group::1 SS (Q K^T)")) return 1;
     if (run<1, 1>(res, "cta_group::1 TS (P V)")) return 1;
+    if (run<1, 0, 64>(res, "cta_group::1 SS, N = 64")) return 1;
+    if (run<1, 0, 256>(res, "cta_group::1 SS, N = 256")) return 1;
     if (run<2, 0>(res, "cta_group::2 SS (Q K^T)")) return 1;
     if (run<2, 1>(res, "cta_group::2 TS (P V)")) return 1;
     return 0;
