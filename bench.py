@@ -432,22 +432,28 @@ def measure(args, cfg_name, rank, world, device, headline):
 
     with torch.cuda.stream(stream):
         # ---- prompt initialisation (the bulk form of cb_update), timed on its own: the tables start empty each time
-        bulk_ms = []
-        for rep in range(3):
-            cb.cb_reset()
-            stream.synchronize()
-            e0.record(stream)
-            cb.cb_update_bulk(toks_d, zeros_d, prefill_d)
-            e1.record(stream)
-            stream.synchronize()
-            bulk_ms.append(e0.elapsed_time(e1))
-    windows = float(np.sum(np.maximum(prefill.astype(np.int64) - cfg.LL - cfg.FL + 1, 0)))
+        # with scratch attached (the order-free path) and without (warps by leader); the last run leaves the tables filled
+        windows = float(np.sum(np.maximum(prefill.astype(np.int64) - cfg.LL - cfg.FL + 1, 0)))
+        bulk_ms, bulk_plain_ms = [], []
+        for with_scratch, acc in ((False, bulk_plain_ms), (True, bulk_ms)):
+            scratch_bytes = cb.cb_bulk_scratch_attach(int(windows) if with_scratch else 0)
+            for rep in range(3):
+                cb.cb_reset()
+                stream.synchronize()
+                e0.record(stream)
+                cb.cb_update_bulk(toks_d, zeros_d, prefill_d)
+                e1.record(stream)
+                stream.synchronize()
+                acc.append(e0.elapsed_time(e1))
+        cb.cb_bulk_scratch_attach(0)
     entry_bytes = (cfg.LL + 1 + cfg.FC * (cfg.FL + 1)) * 4
     bulk_bytes = windows * (entry_bytes + (cfg.FL + 2) * 4)
     bulk_t = float(np.median(bulk_ms)) * 1e-3
     bulk = {"ms": 1e3 * bulk_t, "windows": windows, "windows_per_s": windows / bulk_t, "algorithmic_bytes": bulk_bytes,
             "bytes_per_window": entry_bytes + (cfg.FL + 2) * 4, "gbs": bulk_bytes / bulk_t / 1e9,
-            "frac_of_hbm": bulk_bytes / bulk_t / 1e9 / pk["hbm_gbs"]}
+            "frac_of_hbm": bulk_bytes / bulk_t / 1e9 / pk["hbm_gbs"], "scratch_bytes": scratch_bytes,
+            "path": "order-free (scratch attached: one thread per window, one warp per distinct leader)",
+            "ms_without_scratch": float(np.median(bulk_plain_ms))}
 
     frozen_info, ft = None, None
     if args.frozen > 0:

@@ -118,10 +118,31 @@ cb_status cb_update(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, cons
  * cb_update for long runs of new tokens (Section 3.3: the dynamic table is initialised with a sliding window over the
  * prompt).  Same arguments, same resulting tables, clocks and counters as cb_update; the work of one sequence is spread
  * over many warps where that cannot change the result (no leader can be evicted during the run: leaders stored + windows
- * <= LC, and at least 64 windows), and done by one warp in order otherwise.  Two launches.
+ * <= LC, and at least 64 windows), and done by one warp in order otherwise.  Two launches (seven with scratch attached,
+ * see below).  CB_CNT_FOLLOWER_EVICTIONS counts the followers this call displaced from the lists; on the order-free path
+ * a follower that the run itself would have stored and displaced again is never stored and so is not counted.
  */
 cb_status cb_update_bulk(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* n_old,
                          const int32_t* n_new, void* stream);
+
+/*
+ * Scratch memory for the order-free path of cb_update_bulk.  After a run in which no leader can be evicted, and under the
+ * reading that re-inserting a stored follower refreshes it (the default), a leader's stamp is that of its last window and its
+ * followers are the FC distinct ones touched last (Section 3.1: both lists are least-recently-used lists), whatever the
+ * order of the windows.  With scratch attached, the sequences of a call whose runs qualify (as above) and fit the scratch,
+ * taken in batch order, are reduced that way: one thread per window, then one warp per distinct leader.  The resulting
+ * tables and clocks are those of cb_update; which place a follower or an entry takes inside the table may differ, which no
+ * call reports.
+ *   cb_bulk_scratch_bytes    HOST out: bytes for calls whose qualifying runs hold up to max_windows windows in total
+ *                            (about 84 to 164 bytes per window: two hash tables of the next power of two >= 2 * max_windows
+ *                            slots); cfg->batch sizes a small per-sequence array.
+ *   cb_bulk_scratch_attach   dev_scratch: DEVICE, 256-byte aligned, `bytes` long, owned by the caller and to be kept while
+ *                            attached; its content need not be initialised and is overwritten by every cb_update_bulk call.
+ *                            NULL detaches.  Calls on one context that use it must not overlap.
+ * Errors: CB_ERR_INVALID_ARG (null, misaligned, too small for any table).
+ */
+cb_status cb_bulk_scratch_bytes(const cb_config* cfg, int64_t max_windows, size_t* bytes);
+cb_status cb_bulk_scratch_attach(cb_ctx* ctx, void* dev_scratch, size_t bytes);
 
 /*
  * Draft-tree growth (Section 3.2).

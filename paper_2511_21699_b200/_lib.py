@@ -23,7 +23,8 @@ COUNTER_NAMES = ["inserts", "leader_evictions", "follower_evictions", "queries",
 EXPORTS = ["cb_workspace_bytes", "cb_create", "cb_destroy", "cb_reset", "cb_update", "cb_draft_tree", "cb_update_draft_tree",
            "cb_tree_attn", "cb_accept", "cb_table_dump", "cb_table_load", "cb_poll_status", "cb_launch_count",
            "cb_status_str", "cb_accept_static", "cb_kv_commit", "cb_frozen_bytes", "cb_frozen_load", "cb_frozen_dump",
-           "cb_frozen_attach", "cb_frozen_build_bytes", "cb_frozen_build", "cb_tree_add_branches", "cb_update_bulk", "cb_debug_build"]
+           "cb_frozen_attach", "cb_frozen_build_bytes", "cb_frozen_build", "cb_tree_add_branches", "cb_update_bulk", "cb_debug_build",
+           "cb_bulk_scratch_bytes", "cb_bulk_scratch_attach"]
 
 
 class CbConfigC(C.Structure):
@@ -65,6 +66,8 @@ def load():
     L.cb_reset.argtypes = [vp, vp, vp]
     L.cb_update.argtypes = [vp, vp, i64, vp, vp, vp]
     L.cb_update_bulk.argtypes = [vp, vp, i64, vp, vp, vp]
+    L.cb_bulk_scratch_bytes.argtypes = [C.POINTER(CbConfigC), i64, C.POINTER(C.c_size_t)]
+    L.cb_bulk_scratch_attach.argtypes = [vp, vp, C.c_size_t]
     L.cb_draft_tree.argtypes = [vp, vp, i64, vp, vp, vp, vp, vp, vp, vp]
     L.cb_update_draft_tree.argtypes = [vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp]
     L.cb_tree_add_branches.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp]

@@ -171,6 +171,22 @@ class Cacheback:
         _check(self.lib.cb_update_bulk(self._h, _ptr(tokens, torch.int32), tokens.stride(0), _ptr(n_old, torch.int32),
                                        _ptr(n_new, torch.int32), _stream(stream)), "cb_update_bulk")
 
+    def cb_bulk_scratch_attach(self, max_windows):
+        """Allocates and attaches scratch for the order-free path of cb_update_bulk (runs of up to max_windows windows in
+        total per call); 0 or None detaches.  The buffer is kept alive by this object."""
+        if not max_windows:
+            _check(self.lib.cb_bulk_scratch_attach(self._h, None, 0), "cb_bulk_scratch_attach")
+            self._bulk_scratch = None
+            return 0
+        nbytes = C.c_size_t(0)
+        _check(self.lib.cb_bulk_scratch_bytes(C.byref(self.cfg), C.c_int64(int(max_windows)), C.byref(nbytes)), "cb_bulk_scratch_bytes")
+        with torch.cuda.device(self.device):
+            buf = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=self.device)
+        ptr = (buf.data_ptr() + 255) // 256 * 256
+        _check(self.lib.cb_bulk_scratch_attach(self._h, C.c_void_p(ptr), C.c_size_t(nbytes.value)), "cb_bulk_scratch_attach")
+        self._bulk_scratch = buf
+        return nbytes.value
+
     def alloc_tree(self):
         B, T = self.cfg.batch, self.cfg.max_nodes
         i32 = dict(dtype=torch.int32, device=self.device)

@@ -95,6 +95,8 @@ struct cb_ctx {
     unsigned long long* d_rowmax;    // [batch * max_nodes] packed (value, index) maxima, zero between calls
     uint32_t* d_ticket;     // [batch] CTAs-finished counters, zero between calls
     uint32_t* d_bulk_plan;  // [batch][4] per-sequence plan of cb_update_bulk
+    void* bulk_scratch;     // caller's scratch for the order-free path of cb_update_bulk (cb_bulk_scratch_attach), or null
+    uint32_t bulk_slots;    // hash slots that fit it (a power of two)
     size_t guard_off[CB_MAX_GUARDS];
     int n_guards;
     float* d_attn_part;     // partial outputs of units shared between CTAs

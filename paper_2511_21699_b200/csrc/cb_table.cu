@@ -271,7 +271,7 @@ __global__ void __launch_bounds__(128) cb_update_kernel(CbTables t, int B, const
 // (atomicAdd hands out entry ids) and the index, whose slots are claimed with atomicCAS; an entry is complete before its
 // index word is published.  A plan kernel takes that decision once per sequence, before any warp changes the table;
 // sequences that do not qualify (short runs, possible eviction) are done by their first warp alone, in order.
-struct BulkPlan { uint32_t parallel, clock0, first, nwin; };
+struct BulkPlan { uint32_t parallel, clock0, first, nwin; };   // parallel: 0 one warp in order, 1 warps by leader, 2 order-free path (cb_bulk_free.cuh)
 
 __global__ void cb_bulk_plan_kernel(CbTables t, int B, const int32_t* __restrict__ n_old, const int32_t* __restrict__ n_new,
                                     BulkPlan* plan) {
@@ -361,6 +361,7 @@ __global__ void __launch_bounds__(256) cb_update_bulk_kernel(CbTables t, int B, 
     if (b >= B) return;
     const CbSeq s = cb_seq(t, b);
     const BulkPlan pl = plan[b];
+    if (pl.parallel == 2u) return;                              // done by the order-free kernels
     const int32_t* row = tokens + (size_t)b * row_stride;
     TblCounters cnt = {0, 0, 0, 0};
     if (!pl.parallel) {
@@ -445,6 +446,12 @@ __global__ void __launch_bounds__(256) cb_update_bulk_kernel(CbTables t, int B, 
         if (cnt.maxprobe) atomicMax(&counters[CB_CNT_MAX_PROBE], (unsigned long long)cnt.maxprobe);
     }
 }
+
+}  // namespace
+
+#include "cb_bulk_free.cuh"
+
+namespace {
 
 // ---------------------------------------------------------------------------------------------------
 // Draft-tree expansion: one CTA per sequence, one warp per frontier leaf ("branch") for the lookups.
@@ -721,7 +728,26 @@ extern "C" cb_status cb_update_bulk(cb_ctx* ctx, const int32_t* tokens, int64_t 
     int wps = 1;
     while (wps < 256 && (long long)B * wps * 2 <= (long long)ctx->num_sms * 64) wps *= 2;
     BulkPlan* plan = reinterpret_cast<BulkPlan*>(ctx->d_bulk_plan);
-    CB_CUDA(cb_launch_pdl(cb_bulk_plan_kernel, dim3((B + 127) / 128), dim3(128), 0, (cudaStream_t)stream, ctx->tables, B, n_old, n_new, plan));
+    const bool free_path = ctx->bulk_scratch && B <= kBulkFreeMaxBatch && ctx->tables.refresh;
+    if (free_path) {
+        // order-free path for the sequences that qualify and fit the attached scratch; the kernel below does the others
+        const BulkFreeView v = bulk_free_view(ctx->bulk_scratch, ctx->bulk_slots, B);
+        const cudaStream_t st = (cudaStream_t)stream;
+        const unsigned blocks = (unsigned)std::min<long long>((long long)v.S / 256, (long long)ctx->num_sms * 8);
+        const unsigned wide = (unsigned)std::min<long long>((long long)v.S / 256, (long long)ctx->num_sms * 32);   // one item per thread, or a few
+        CB_CUDA(cb_launch_pdl(cb_bulk_free_plan_kernel, dim3(1), dim3(1024), 0, st, ctx->tables, B, n_old, n_new, plan, v, ctx->d_counters));
+        CB_CUDA(cb_launch_pdl(cb_bulk_free_clear_kernel, dim3(wide), dim3(256), 0, st, v));
+        CB_CUDA(cb_launch_pdl(cb_bulk_free_reduce_kernel, dim3(wide), dim3(256), 0, st, ctx->tables, B, tokens, row_stride, (const BulkPlan*)plan, v,
+                              ctx->d_status));
+        CB_CUDA(cb_launch_pdl(cb_bulk_free_ranges_kernel, dim3(wide), dim3(256), 0, st, v));
+        CB_CUDA(cb_launch_pdl(cb_bulk_free_scatter_kernel, dim3(wide), dim3(256), 0, st, v));
+        CB_CUDA(cb_launch_pdl(cb_bulk_free_apply_kernel, dim3(blocks), dim3(256), 0, st, ctx->tables, B, tokens, row_stride, (const BulkPlan*)plan, v,
+                              ctx->d_status, ctx->d_counters));
+        cb_count_launch(6);
+    } else {
+        CB_CUDA(cb_launch_pdl(cb_bulk_plan_kernel, dim3((B + 127) / 128), dim3(128), 0, (cudaStream_t)stream, ctx->tables, B, n_old, n_new, plan));
+        cb_count_launch(1);
+    }
     const long long warps = (long long)B * wps;
     // kept entries per warp: four, fewer where 96 KB of shared memory per CTA (8 warps) do not hold that many
     const size_t way_bytes = ((size_t)ctx->tables.E + 4) * 4;
@@ -738,7 +764,30 @@ extern "C" cb_status cb_update_bulk(cb_ctx* ctx, const int32_t* tokens, int64_t 
     }
     CB_CUDA(cb_launch_pdl(cb_update_bulk_kernel, dim3((unsigned)((warps + 7) / 8)), dim3(256), smem, (cudaStream_t)stream, ctx->tables, B, wps, n_ways,
                           tokens, row_stride, n_old, n_new, (const BulkPlan*)plan, ctx->d_status, ctx->d_counters));
-    cb_count_launch(2);
+    cb_count_launch(1);
+    return CB_OK;
+}
+
+extern "C" cb_status cb_bulk_scratch_bytes(const cb_config* cfg, int64_t max_windows, size_t* bytes) {
+    CB_CHECK_ARG(cfg && bytes && cfg->batch >= 1 && max_windows >= 1 && max_windows <= (int64_t)1 << 29);
+    uint32_t S = 2048;
+    while ((int64_t)S < 2 * max_windows) S <<= 1;
+    *bytes = bulk_free_layout(S, cfg->batch).total;
+    return CB_OK;
+}
+
+extern "C" cb_status cb_bulk_scratch_attach(cb_ctx* ctx, void* dev_scratch, size_t bytes) {
+    CB_CHECK_ARG(ctx);
+    ctx->bulk_scratch = nullptr;
+    ctx->bulk_slots = 0;
+    if (!dev_scratch) return CB_OK;
+    CB_CHECK_ARG((reinterpret_cast<uintptr_t>(dev_scratch) & 255u) == 0);
+    // the largest power-of-two slot count whose layout fits
+    uint32_t S = 0;
+    for (uint32_t c = 2048; c != 0 && c <= (1u << 30) && bulk_free_layout(c, ctx->cfg.batch).total <= bytes; c <<= 1) S = c;
+    CB_CHECK_ARG(S != 0);
+    ctx->bulk_scratch = dev_scratch;
+    ctx->bulk_slots = S;
     return CB_OK;
 }
 

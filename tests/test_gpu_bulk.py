@@ -14,12 +14,20 @@ pytestmark = pytest.mark.gpu
 
 @pytest.mark.parametrize("name,flags", [("c1_tiny", 0), ("c2_7b", 0), ("c2_7b", 1), ("c3_8b_gqa", 0), ("c4_13b_turns", 0),
                                         ("p_tuned", 0), ("p_fc40_evict", 0), ("c1_evict256", 0), ("c5_70b_long", 0)])
-def test_bulk_prompt_then_incremental_then_draft(oracle, name, flags):
+@pytest.mark.parametrize("scratch", ["none", "all", "some"])
+def test_bulk_prompt_then_incremental_then_draft(oracle, name, flags, scratch):
+    """scratch: "all" attaches scratch that holds every sequence's run (the order-free path where a run qualifies), "some"
+    scratch for about half of the batch's windows (the rest takes the other paths in the same call)."""
     from paper_2511_21699_b200 import Cacheback
     cfg = W.get_config(name)
     prob = Problem(cfg)
     B, T = cfg.batch, cfg.max_nodes
+    if scratch == "some" and B < 4:
+        pytest.skip("one sequence: nothing to split")
     cb = Cacheback.from_config(cfg, flags=flags)
+    if scratch != "none":
+        total = int(np.sum(prob.prefill))
+        cb.cb_bulk_scratch_attach(total if scratch == "all" else max(total // 2, 1024))
     check = list(range(B)) if B <= 8 else [0, 1, B // 2, B - 1]
     otabs = {b: oracle.OracleTable(cfg.LL, cfg.FL, cfg.LC, cfg.FC, refresh_on_reinsert=not (flags & 1)) for b in check}
     toks_d = dev(prob.toks)
@@ -64,7 +72,7 @@ def test_bulk_prompt_then_incremental_then_draft(oracle, name, flags):
 
 
 def test_bulk_equals_sequential_call_on_a_prompt():
-    """The same prompt through cb_update and through cb_update_bulk: identical dumps (the times are printed; the benchmark reports them)."""
+    """The same prompt through cb_update, cb_update_bulk and cb_update_bulk with scratch: identical dumps (the times are printed; the benchmark reports them)."""
     from paper_2511_21699_b200 import Cacheback
     cfg = W.get_config("c2_7b")
     prob = Problem(cfg)
@@ -73,10 +81,12 @@ def test_bulk_equals_sequential_call_on_a_prompt():
     n = dev(prob.prefill)
     times = {}
     dumps = {}
-    for kind in ("seq", "bulk"):
+    for kind in ("seq", "bulk", "bulk_scratch"):
         best = 1e9
         for rep in range(3):
             cb = Cacheback.from_config(cfg)
+            if kind == "bulk_scratch":
+                cb.cb_bulk_scratch_attach(int(prob.prefill[0]))
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             (cb.cb_update if kind == "seq" else cb.cb_update_bulk)(toks_d, zero, n)
@@ -85,5 +95,5 @@ def test_bulk_equals_sequential_call_on_a_prompt():
             best = min(best, e0.elapsed_time(e1))
         times[kind] = best
         dumps[kind] = cb.cb_table_dump(0)
-    assert dumps["seq"] == dumps["bulk"]
-    print("prompt of %d tokens: sequential %.3f ms, bulk %.3f ms" % (int(prob.prefill[0]), times["seq"], times["bulk"]))
+    assert dumps["seq"] == dumps["bulk"] == dumps["bulk_scratch"]
+    print("prompt of %d tokens: sequential %.3f ms, bulk %.3f ms, bulk with scratch %.3f ms" % (int(prob.prefill[0]), times["seq"], times["bulk"], times["bulk_scratch"]))
