@@ -194,14 +194,15 @@ __global__ void __launch_bounds__(256) cb_bulk_free_reduce_kernel(CbTables t, in
     }
 }
 
-// 2. every leader takes its range of the group array (one atomicAdd per warp: the ranges of its leaders lie side by side)
+// 2. every leader takes its range of the group array (one atomicAdd per block and 256 slots: their ranges lie side by side)
 __global__ void __launch_bounds__(256) cb_bulk_free_ranges_kernel(BulkFreeView v) {
     CB_PDL_ENTRY();
     if (v.hdr->m_total == 0) return;
-    const uint32_t S = v.hdr->s_eff;
-    const int lane = threadIdx.x & 31;
-    for (uint32_t i0 = (blockIdx.x * blockDim.x + threadIdx.x) & ~31u; i0 < S; i0 += gridDim.x * blockDim.x) {
-        const uint32_t i = i0 + lane;                           // S is a multiple of 32
+    const uint32_t S = v.hdr->s_eff;                             // a multiple of 256
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __shared__ uint32_t s_tot[8], s_start;
+    for (uint32_t i0 = blockIdx.x * 256u; i0 < S; i0 += gridDim.x * 256u) {
+        const uint32_t i = i0 + threadIdx.x;
         const uint32_t n = v.lrep[i] != 0ull ? v.lcount[i] : 0u;
         uint32_t incl = n;
 #pragma unroll
@@ -209,11 +210,16 @@ __global__ void __launch_bounds__(256) cb_bulk_free_ranges_kernel(BulkFreeView v
             const uint32_t up = __shfl_up_sync(CB_FULL, incl, o);
             if (lane >= o) incl += up;
         }
-        const uint32_t total = __shfl_sync(CB_FULL, incl, 31);
-        uint32_t start = 0;
-        if (lane == 0 && total) start = atomicAdd(&v.hdr->cursor, total);
-        start = __shfl_sync(CB_FULL, start, 0);
-        if (n) { v.lbase[i] = start + incl - n; v.lfill[i] = 0u; }
+        if (lane == 31) s_tot[warp] = incl;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t total = 0;
+            for (int k = 0; k < 8; ++k) { const uint32_t c = s_tot[k]; s_tot[k] = total; total += c; }
+            s_start = total ? atomicAdd(&v.hdr->cursor, total) : 0u;
+        }
+        __syncthreads();
+        if (n) { v.lbase[i] = s_start + s_tot[warp] + incl - n; v.lfill[i] = 0u; }
+        __syncthreads();                                         // the shared words are rewritten by the next round
     }
 }
 
@@ -262,7 +268,63 @@ __global__ void __launch_bounds__(256) cb_bulk_free_apply_kernel(CbTables t, int
         }
         // what this lane's leader still needs at the end: its new entry's index word and the slot found free for it
         uint32_t my_word = 0, my_free = 0xFFFFFFFFu;
-        uint32_t todo = __ballot_sync(CB_FULL, occ);
+        // ---- per lane: the common case of a prompt, a leader that is not in the table yet and has a few followers, is done
+        // by its lane alone (32 leaders side by side instead of one after the other): the home bucket shows no index word
+        // with the leader's tag and has room, so the leader is absent and its word goes there; the lane takes an entry and
+        // writes it.  Every other case (a word with the tag, a full bucket, many followers) is left to the whole warp below.
+        bool handled = false;
+        if (occ && my_n <= (uint32_t)min(t.FC, 8)) {
+            const int b = (int)(my_rep >> 32);
+            const CbSeq s = cb_seq(t, b);
+            const uint32_t bucket = cb_hash_bucket(my_h, t.nslots), tag = cb_hash_tag(my_h);
+            const uint4* bp = reinterpret_cast<const uint4*>(s.index + (size_t)bucket * 32);
+            uint32_t w[32];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { const uint4 x = __ldcg(bp + q); w[4 * q] = x.x; w[4 * q + 1] = x.y; w[4 * q + 2] = x.z; w[4 * q + 3] = x.w; }
+            bool tagged = false, has_empty = false;
+            int first_free = -1;
+#pragma unroll
+            for (int q = 0; q < 32; ++q) {
+                const bool emp = w[q] == CB_IDX_EMPTY, tomb = w[q] == CB_IDX_TOMB;
+                has_empty = has_empty || emp;
+                if ((emp || tomb) && first_free < 0) first_free = q;
+                tagged = tagged || (!emp && !tomb && (w[q] >> CB_EID_BITS) == tag);
+            }
+            if (!tagged && has_empty && my_gbase + my_n <= v.W) {
+                const uint32_t got = atomicAdd(&s.hdr[1], 1u);
+                if (got < (uint32_t)t.LC) {                     // anything else is excluded by the plan
+                    const uint32_t clock0 = plan[b].clock0;
+                    const int32_t* row = tokens + (size_t)b * row_stride;
+                    uint32_t* e = s.entries + (size_t)got * t.E;
+                    for (int j = 0; j < t.LL; ++j) e[j] = (uint32_t)my_k[j];
+                    // loads first, level by level, so that the followers' round trips overlap
+                    uint32_t ps[8], fl[8], fp[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) ps[j] = (uint32_t)j < my_n ? v.group[my_gbase + j] : 0u;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        fl[j] = (uint32_t)j < my_n ? v.plast[ps[j]] : 0u;
+                        fp[j] = (uint32_t)j < my_n ? (uint32_t)v.prep[ps[j]] - 1u : 0u;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if ((uint32_t)j >= my_n) break;
+                        int32_t ft[CB_MAX_FL];
+#pragma unroll
+                        for (int f = 0; f < CB_MAX_FL; ++f) ft[f] = f < t.FL ? row[fp[j] + t.LL + f] : 0;
+                        e[t.LL + j] = clock0 + fl[j];
+#pragma unroll
+                        for (int f = 0; f < CB_MAX_FL; ++f) if (f < t.FL) e[t.LL + t.FC + j * t.FL + f] = (uint32_t)ft[f];
+                    }
+                    for (int f = (int)my_n; f < t.FC; ++f) e[t.LL + f] = 0u;
+                    s.lstamp[got] = clock0 + my_last;
+                    my_word = (tag << CB_EID_BITS) | got;
+                    my_free = bucket * 32u + (uint32_t)first_free;
+                    handled = true;
+                }
+            }
+        }
+        uint32_t todo = __ballot_sync(CB_FULL, occ && !handled);
         while (todo) {
             const int src = __ffs(todo) - 1;
             todo &= todo - 1;
