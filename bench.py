@@ -58,16 +58,22 @@ def parse(argv=None):
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one cb_attn_tc_kernel launch with full trees, from the ncu
 # captures summarised under profiles/.  Reported only while the kernel sources still hash to the captured ones; after any
 # change to them the figure is stale and `traffic` is null until the capture is redone.
-ATTN_TRAFFIC = {"sources_sha1": "940d4a8002e5bcb4876bd7445ef665e14f2a13aa",
-                "bytes_per_launch": {"c2_7b": 70.37e6, "c3_8b_gqa": 558.2e6, "c4_13b_turns": 2768.5e6},
-                "source": {"c2_7b": "profiles/cb_attn_tc_kernel_c2_7b.md", "c3_8b_gqa": "profiles/cb_attn_tc_kernel_c3_c4.md",
-                           "c4_13b_turns": "profiles/cb_attn_tc_kernel_c3_c4.md"}}
+ATTN_TRAFFIC = {"sources_sha1": "b4b33f08ee5ad9b1284c566a679382da21a60dba",
+                "bytes_per_launch": {"c2_7b": 70.2e6, "c3_8b_gqa": 557.8e6, "c4_13b_turns": 2768.8e6},
+                "source": {k: "profiles/cb_attn_tc_kernel_c2_c3_c4_c5b8.md" for k in ("c2_7b", "c3_8b_gqa", "c4_13b_turns")},
+                # config 5 holds 25 GB and runs 20 ms per launch: too large to capture.  The same shape at batch 8 was captured
+                # twice (1,413.9 and 1,688.3 MB per launch); keys and values are streamed per sequence, so the traffic is taken
+                # to grow with the batch: mean x 128 / 8.
+                "scaled": {"c5_70b_long": (0.5 * (1413.9e6 + 1688.3e6) * 16.0,
+                                           "profiles/cb_attn_tc_kernel_c2_c3_c4_c5b8.md: c5_70b_b8 (same shape, batch 8), mean of two captures "
+                                           "x 16 sequences' worth; not a capture of this workload")}}
+ATTN_SOURCES = ("cb_attn_tc.cu", "cb_tc_dev.cuh", "cb_attn_pair.cuh", "cb_attn.cuh", "cb_attn.cu")
 
 
 def attn_sources_sha1():
     import hashlib
     h = hashlib.sha1()
-    for f in ("cb_attn_tc.cu", "cb_attn.cuh", "cb_attn.cu"):
+    for f in ATTN_SOURCES:
         with open(os.path.join(ROOT, "paper_2511_21699_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()
@@ -582,6 +588,8 @@ def measure(args, cfg_name, rank, world, device, headline):
     if ATTN_TRAFFIC["sources_sha1"] == attn_sources_sha1() and cfg_name in ATTN_TRAFFIC["bytes_per_launch"]:
         traffic = ATTN_TRAFFIC["bytes_per_launch"][cfg_name]
         traffic_source = ATTN_TRAFFIC["source"][cfg_name] + " (ncu dram__bytes_read.sum + dram__bytes_write.sum; kernel sources hash-matched)"
+    elif ATTN_TRAFFIC["sources_sha1"] == attn_sources_sha1() and cfg_name in ATTN_TRAFFIC["scaled"]:
+        traffic, traffic_source = ATTN_TRAFFIC["scaled"][cfg_name]
     roof_full.update({"traffic": traffic, "traffic_source": traffic_source,
                       "kernel": "cb_tree_attn (attention kernel, plus its merge pass where the launch is not in cluster mode)"})
     acc_bytes_full, acc_bytes_dr = float(B * T) * cfg.vocab * 4, float(np.sum(nn_mean)) * cfg.vocab * 4
