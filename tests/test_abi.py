@@ -51,3 +51,24 @@ def test_frozen_table_sizes_and_argument_checks_need_no_gpu():
                 _lib.CbFrozenConfigC(1, 3, (1 << 20) + 1, 4)):
         assert lib.cb_frozen_bytes(ctypes.byref(bad), ctypes.byref(n)) == 1
     assert lib.cb_frozen_attach(None, ctypes.byref(cfg), None, 0) == 1            # no context
+
+
+def test_bulk_scratch_sizes_and_argument_checks_need_no_gpu():
+    """Two hash tables of the next power of two >= 2 * windows slots at 40 bytes a slot, plus 4 bytes per window place."""
+    from paper_2511_21699_b200 import _lib
+    lib = _lib.load()
+    cfg = _lib.CbConfigC(128, 3, 5, 65536, 8, 128, 32, 16, 32000, 64, 8, 128, 16, 0)
+    n = ctypes.c_size_t(0)
+    last = 0
+    for windows in (1, 1000, 4096, 4097, 127459, 4193536):
+        assert lib.cb_bulk_scratch_bytes(ctypes.byref(cfg), windows, ctypes.byref(n)) == 0
+        slots = 2048
+        while slots < 2 * windows:
+            slots *= 2
+        assert 42 * slots <= n.value <= 42 * slots + 16 * 256 + (cfg.batch + 1) * 4 + 64, (windows, n.value)
+        assert n.value >= last
+        last = n.value
+    assert lib.cb_bulk_scratch_bytes(ctypes.byref(cfg), 0, ctypes.byref(n)) == 1
+    assert lib.cb_bulk_scratch_bytes(ctypes.byref(cfg), (1 << 29) + 1, ctypes.byref(n)) == 1
+    assert lib.cb_bulk_scratch_bytes(None, 16, ctypes.byref(n)) == 1
+    assert lib.cb_bulk_scratch_attach(None, None, 0) == 1                           # no context
