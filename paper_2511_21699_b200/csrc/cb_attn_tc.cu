@@ -6,11 +6,12 @@
 // ring; eight 16-token pages per tile, fetched page by page with TMA through the block table).
 //
 // Warp roles (384 threads, three warpgroups):
-//   warp 0        TMA producer for K/V: runs ahead across unit boundaries, limited only by the ring
+//   warp 0        TMA producer for the K tiles (warp 3 for the V tiles): runs ahead across unit boundaries, limited only
+//                 by the ring
 //   warp 1        MMA issuer (one lane): S = Q K^T into TMEM, then O += P V with P read from TMEM;
 //                 owns the TMEM allocation (S0, S1, O0, O1: 4 x 128 columns)
 //   warp 2        TMA loader for the query tiles of each unit
-//   warp 3        writes the zero rows of padding nodes (node >= n_nodes)
+//   warp 3        writes the zero rows of padding nodes (node >= n_nodes), then TMA producer for the V tiles
 //   warps 4..7    softmax warpgroup 0, warps 8..11 softmax warpgroup 1: one thread per query row; S from
 //                 TMEM to registers, fp32 online softmax in the log2 domain with lazy rescaling of O,
 //                 P written back to TMEM as packed bf16 over S; epilogue of the unit
@@ -150,34 +151,52 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
 
     if (warp < 4) {
         reg_dealloc<120>();
-        if (warp == 0) {
-            // ------------------------------------------------------------------ K/V producer
-            constexpr int NB = 8 * C::DB;                    // boxes (16 keys x 64 dims) per tile
-            const bool active = lane < 2 * NB;
-            const bool isV = lane >= NB;
-            const int within = lane % NB, j = within % 8, dblk = within / 8;
-            uint32_t seq = 0;
+        if (warp == 0 || warp == 3) {
+            // ------------------------------------------------------------------ K/V producers: warp 0 the K tiles, warp 3 the V tiles
+            // A tile is 8 * DB boxes of 16 keys x 64 dims, one copy instruction each, and the copies of one warp instruction
+            // are issued one after the other: two warps issue the two tiles of a key tile side by side.
+            const bool isV = warp == 3;
+            if (isV) {
+                // rows of padding nodes (node >= n_nodes) are written as zeros: once, before the first V tile is wanted
+                const int per_row = p.Hq * D / 8;            // 16-byte chunks per node row
+                for (int idx = cta; idx < p.B * p.T; idx += gridDim.x) {
+                    const int b = idx / p.T, node = idx % p.T;
+                    const int n = min(max(p.n_nodes[b], 0), p.T);
+                    if (node < n) continue;
+                    uint4* op = reinterpret_cast<uint4*>(p.out + (size_t)idx * p.Hq * D);
+                    for (int k = lane; k < per_row; k += 32) op[k] = make_uint4(0, 0, 0, 0);
+                    if (p.lse) for (int h = lane; h < p.Hq; h += 32) p.lse[((size_t)b * p.Hq + h) * p.T + node] = 0.f;
+                }
+            }
+            constexpr int NB = 8 * C::DB;                    // boxes per tile
+            const bool active = lane < NB;
+            const int j = lane % 8, dblk = (lane % NB) / 8;
+            uint32_t seq = isV ? 1u : 0u;                    // K and V tiles alternate in the ring
             bool ok = true;
             const uint64_t pol = l2_evict_first_policy();
             while (ok && wk.next(p, &u)) {
                 const int npages = (u.ctx + p.P - 1) / p.P, nct = u.tiles - 1;
                 const int32_t* bt = p.block_table + (size_t)u.b * p.max_pages;
-                for (int i = u.t0; i < u.t1; ++i) {
+                // The page number of a lane's box comes from the block table: a memory round trip that the copy depends on.
+                // It is fetched one tile ahead, so that it is under way while this tile's copies are issued and waited for.
+                auto page_of = [&](int i) {
                     int page = p.num_pages;                  // out of range: the copy fills zeros
                     if (active && i < nct) {
                         const int pidx = i * (CB_KT / 16) + j;
-                        if (pidx < npages) {
-                            page = bt[pidx];
-                            if (!cb_dbg_in(page, p.num_pages, p.status)) page = p.num_pages;   // the copy then fills zeros
-                        }
+                        if (pidx < npages) page = bt[pidx];
                     }
-                    const uint32_t ks = seq % C::NSLOT, vs = (seq + 1) % C::NSLOT;
-                    if (seq >= (uint32_t)C::NSLOT && !(ok = mbar_wait(bar_free(ks), (seq / C::NSLOT - 1) & 1, s_abort, p.status))) break;
-                    if (seq + 1 >= (uint32_t)C::NSLOT && !(ok = mbar_wait(bar_free(vs), ((seq + 1) / C::NSLOT - 1) & 1, s_abort, p.status))) break;
-                    if (lane == 0) { mbar_expect_tx(bar_full(ks), C::TILE_BYTES); mbar_expect_tx(bar_full(vs), C::TILE_BYTES); }
+                    return page;
+                };
+                int page_next = page_of(u.t0);
+                for (int i = u.t0; i < u.t1; ++i) {
+                    int page = page_next;
+                    if (i + 1 < u.t1) page_next = page_of(i + 1);
+                    if (!cb_dbg_in(page, p.num_pages + 1, p.status)) page = p.num_pages;   // the copy then fills zeros
+                    const uint32_t sl = seq % C::NSLOT;
+                    if (seq >= (uint32_t)C::NSLOT && !(ok = mbar_wait(bar_free(sl), (seq / C::NSLOT - 1) & 1, s_abort, p.status))) break;
+                    if (lane == 0) mbar_expect_tx(bar_full(sl), C::TILE_BYTES);
                     __syncwarp();
                     if (active) {
-                        const uint32_t sl = isV ? vs : ks;
                         const uint32_t dst = sbase + C::OFF_RING + sl * C::TILE_BYTES + dblk * (CB_KT * 128) + j * 2048;
                         if (i < nct) tma_load_4d_hint(dst, isV ? &maps.v_pool : &maps.k_pool, bar_full(sl), dblk * 64, u.kh, 0, page, pol);
                         else tma_load_4d(dst, isV ? &maps.v_tree : &maps.k_tree, bar_full(sl), dblk * 64, u.kh, 16 * j, u.b);
@@ -295,17 +314,6 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                 }
             }
             __syncwarp();
-        } else {
-            // ------------------------------------------------------------------ zero rows of padding nodes
-            const int per_row = p.Hq * D / 8;                // 16-byte chunks per node row
-            for (int idx = cta; idx < p.B * p.T; idx += gridDim.x) {
-                const int b = idx / p.T, node = idx % p.T;
-                const int n = min(max(p.n_nodes[b], 0), p.T);
-                if (node < n) continue;
-                uint4* op = reinterpret_cast<uint4*>(p.out + (size_t)idx * p.Hq * D);
-                for (int k = lane; k < per_row; k += 32) op[k] = make_uint4(0, 0, 0, 0);
-                if (p.lse) for (int h = lane; h < p.Hq; h += 32) p.lse[((size_t)b * p.Hq + h) * p.T + node] = 0.f;
-            }
         }
     } else {
         // ---------------------------------------------------------------------- softmax / correction / epilogue
