@@ -255,6 +255,47 @@ cb_status cb_accept(cb_ctx* ctx, const int32_t* tree_tokens, const int32_t* tree
                     int32_t* target_ids_out, void* stream);
 
 /*
+ * One step's acceptance and the next step's update and draft in one launch (Fig. 2: per sequence the three follow one
+ * another — the emitted tokens extend the sequence, their windows go into the table, the next tree is drafted from it).
+ * Same results, table state, counters and errors as
+ *   cb_accept(tree_*, n_nodes, logits, ..., NULL, n_accept, accept_nodes, out_tokens, target_ids_out);
+ *   tokens[b][seq_len[b] .. seq_len[b] + n_accept[b] + 1) = out_tokens[b][0 .. n_accept[b] + 1);   old = seq_len;   seq_len += n_accept + 1;
+ *   cb_update(tokens, row_stride, old, seq_len);   cb_draft_tree(tokens, row_stride, seq_len, next_*);
+ * At small batch the step saves two kernel boundaries.
+ *   logits .. target_ids_out   as in cb_accept (logits only)
+ *   tokens      int32 [batch, row_stride]  DEVICE, read and written: the emitted tokens are appended
+ *   seq_len     int32 [batch]              DEVICE, read and written: tokens valid per sequence
+ *   next_tokens, next_parent, next_depth, next_mask, next_n_nodes   the next tree, as written by cb_draft_tree; they may be the
+ *               arrays of the verified tree (a sequence's acceptance has read them before its draft writes them)
+ * A sequence whose history has no room for the emitted tokens (seq_len + n_accept + 1 > row_stride) keeps its length, nothing
+ * is appended, the draft is made from the sequence as it is, and CB_ERR_INVALID_ARG is recorded in the device status.  A
+ * sequence with an empty tree (n_nodes = 0) emits nothing.
+ */
+typedef struct cb_accept_draft_args {
+    const void* logits;
+    int32_t logits_dtype;
+    int64_t logits_row_stride;
+    const int32_t* tree_tokens;
+    const int32_t* tree_parent;
+    const int32_t* tree_depth;
+    const int32_t* n_nodes;
+    int32_t* n_accept;
+    int32_t* accept_nodes;
+    int32_t* out_tokens;
+    int32_t* target_ids_out;
+    int32_t* tokens;
+    int64_t row_stride;
+    int32_t* seq_len;
+    int32_t* next_tokens;
+    int32_t* next_parent;
+    int32_t* next_depth;
+    uint32_t* next_mask;
+    int32_t* next_n_nodes;
+} cb_accept_draft_args;
+
+cb_status cb_accept_update_draft_tree(cb_ctx* ctx, const cb_accept_draft_args* args, void* stream);
+
+/*
  * KV commit of the accepted path (Section 3.2: the draft tokens and the pending token are the tokens of the
  * verification pass that have no cached K/V; once a branch is accepted its tokens are ordinary context for the next
  * step).  For every sequence b with m = n_accept[b], the tree root (node 0) and the accepted nodes accept_nodes[b, 0..m),

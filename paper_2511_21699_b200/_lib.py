@@ -24,7 +24,7 @@ EXPORTS = ["cb_workspace_bytes", "cb_create", "cb_destroy", "cb_reset", "cb_upda
            "cb_tree_attn", "cb_accept", "cb_table_dump", "cb_table_load", "cb_poll_status", "cb_launch_count",
            "cb_status_str", "cb_accept_static", "cb_kv_commit", "cb_frozen_bytes", "cb_frozen_load", "cb_frozen_dump",
            "cb_frozen_attach", "cb_frozen_build_bytes", "cb_frozen_build", "cb_tree_add_branches", "cb_update_bulk", "cb_debug_build",
-           "cb_bulk_scratch_bytes", "cb_bulk_scratch_attach"]
+           "cb_bulk_scratch_bytes", "cb_bulk_scratch_attach", "cb_accept_update_draft_tree"]
 
 
 class CbConfigC(C.Structure):
@@ -39,6 +39,13 @@ class CbFrozenConfigC(C.Structure):
 class CbKvCommitArgsC(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("k_pool", "v_pool", "block_table", "ctx_len", "k_tree", "v_tree", "n_accept",
                                           "accept_nodes")] + [("max_pages", C.c_int32), ("num_pages", C.c_int32)]
+
+
+class CbAcceptDraftArgsC(C.Structure):
+    _fields_ = [("logits", C.c_void_p), ("logits_dtype", C.c_int32), ("logits_row_stride", C.c_int64)] + \
+               [(n, C.c_void_p) for n in ("tree_tokens", "tree_parent", "tree_depth", "n_nodes", "n_accept", "accept_nodes", "out_tokens",
+                                          "target_ids_out", "tokens")] + [("row_stride", C.c_int64)] + \
+               [(n, C.c_void_p) for n in ("seq_len", "next_tokens", "next_parent", "next_depth", "next_mask", "next_n_nodes")]
 
 
 class CbAttnArgsC(C.Structure):
@@ -72,6 +79,7 @@ def load():
     L.cb_update_draft_tree.argtypes = [vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp]
     L.cb_tree_add_branches.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp]
     L.cb_tree_attn.argtypes = [vp, C.POINTER(CbAttnArgsC), vp]
+    L.cb_accept_update_draft_tree.argtypes = [vp, C.POINTER(CbAcceptDraftArgsC), vp]
     L.cb_kv_commit.argtypes = [vp, C.POINTER(CbKvCommitArgsC), vp]
     L.cb_accept.argtypes = [vp, vp, vp, vp, vp, vp, i32, i64, vp, vp, vp, vp, vp, vp]
     L.cb_accept_static.argtypes = [i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, i64, vp, vp, vp, vp, vp]

@@ -265,6 +265,30 @@ class Cacheback:
                                   _ptr(res["target_ids"], torch.int32), _stream(stream)), "cb_accept")
         return res
 
+    def cb_accept_update_draft_tree(self, tree, logits, tokens, seq_len, next_tree=None, res=None, stream=None):
+        """cb_accept on `tree` and `logits`, the emitted tokens appended to `tokens` (seq_len advanced in place), then cb_update
+        and cb_draft_tree into next_tree (default: the same arrays as `tree`), in one launch."""
+        res = res if res is not None else self.alloc_accept()
+        next_tree = next_tree if next_tree is not None else tree
+        if logits.dtype == torch.float32:
+            dtype = _lib.CB_DTYPE_F32
+        elif logits.dtype == torch.bfloat16:
+            dtype = _lib.CB_DTYPE_BF16
+        else:
+            raise CachebackError("logits must be float32 or bfloat16")
+        if not (logits.is_cuda and logits.dim() == 3 and logits.stride(2) == 1 and logits.stride(0) == logits.shape[1] * logits.stride(1)):
+            raise CachebackError("logits must be [batch, max_nodes, vocab] with a uniform row stride")
+        a = _lib.CbAcceptDraftArgsC(logits.data_ptr(), dtype, logits.stride(1), _ptr(tree["tokens"], torch.int32),
+                                    _ptr(tree["parent"], torch.int32), _ptr(tree["depth"], torch.int32), _ptr(tree["n_nodes"], torch.int32),
+                                    _ptr(res["n_accept"], torch.int32), _ptr(res["accept_nodes"], torch.int32),
+                                    _ptr(res["out_tokens"], torch.int32), _ptr(res["target_ids"], torch.int32),
+                                    _ptr(tokens, torch.int32), tokens.stride(0), _ptr(seq_len, torch.int32),
+                                    _ptr(next_tree["tokens"], torch.int32), _ptr(next_tree["parent"], torch.int32),
+                                    _ptr(next_tree["depth"], torch.int32), _ptr(next_tree["mask"], torch.int32),
+                                    _ptr(next_tree["n_nodes"], torch.int32))
+        _check(self.lib.cb_accept_update_draft_tree(self._h, C.byref(a), _stream(stream)), "cb_accept_update_draft_tree")
+        return res
+
     # ---- helpers ------------------------------------------------------------------------------------
     def cb_frozen_attach(self, frozen):
         """frozen: a FrozenTable (kept alive by this object) or None to detach."""

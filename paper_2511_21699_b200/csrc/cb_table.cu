@@ -5,8 +5,9 @@
 // dense stamp array for the least recently used leader.  Recency is a per-sequence operation counter
 // ("clock"); a leader or follower stamp is the clock value of the operation that last touched it.
 #include <algorithm>
+#include <mutex>
 
-#include "cb_common.cuh"
+#include "cb_accept_dev.cuh"
 
 namespace {
 
@@ -227,7 +228,7 @@ __device__ void tbl_insert(const CbTables& t, const CbSeq& s, int32_t mykey, int
 
 // One warp per sequence; windows are applied in increasing position.
 template <int FETCH>
-__device__ __forceinline__ void update_seq(const CbTables& t, int b, const int32_t* __restrict__ tokens, int64_t row_stride, int n0, int n1,
+__device__ __forceinline__ void update_seq(const CbTables& t, int b, const int32_t* tokens, int64_t row_stride, int n0, int n1,
                                            int lane, uint32_t* status, unsigned long long* counters) {
     const CbSeq s = cb_seq(t, b);
     const int w = t.LL + t.FL;
@@ -471,16 +472,16 @@ struct DraftSmem {
     int32_t* fol;
 };
 
+// The work of the CTA that drafts sequence b, whose history holds L tokens.  upd_n_old >= 0: the windows that the tokens
+// from upd_n_old on complete are inserted first (cb_update_draft_tree and the call that follows an acceptance).  The
+// history may have been extended by this CTA just before (no read-only path to it).
 template <int FETCH>
-__global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, int T, int crt, int max_depth, int NL, int KF,
-                                                       const int32_t* __restrict__ tokens, int64_t row_stride,
-                                                       const int32_t* __restrict__ seq_len, const int32_t* __restrict__ upd_n_old,
-                                                       int32_t* __restrict__ o_tok, int32_t* __restrict__ o_par,
-                                                       int32_t* __restrict__ o_dep, uint32_t* __restrict__ o_mask,
-                                                       int32_t* __restrict__ o_n, uint32_t* status,
-                                                       unsigned long long* counters) {
-    CB_PDL_ENTRY();
-    extern __shared__ int32_t smem[];
+__device__ __forceinline__ void draft_body(const CbTables& t, const CbTables& tf, int T, int crt, int max_depth, int NL, int KF,
+                                           const int32_t* tokens, int64_t row_stride, int b, int L, int upd_n_old,
+                                           int32_t* __restrict__ o_tok, int32_t* __restrict__ o_par,
+                                           int32_t* __restrict__ o_dep, uint32_t* __restrict__ o_mask,
+                                           int32_t* __restrict__ o_n, uint32_t* status,
+                                           unsigned long long* counters, int32_t* smem) {
     DraftSmem S;
     S.tok = smem; S.par = S.tok + T; S.dep = S.par + T;
     S.front = S.dep + T; S.next = S.front + NL; S.pts = S.next + NL;
@@ -489,14 +490,13 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
     S.fol = S.r_nn0 + NL;
     __shared__ int sh_n, sh_nfront, sh_nnext, sh_npts, sh_q, sh_hits, sh_fq, sh_fhits;
 
-    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
     const CbSeq s = cb_seq(t, b);
     const int32_t* row = tokens + (size_t)b * row_stride;
-    const int L = seq_len[b];
-    if (upd_n_old != nullptr) {
+    if (upd_n_old >= 0) {
         // cb_update_draft_tree: the sequence's new windows go into the table first (one warp, in order, exactly as
         // cb_update does), then the whole CTA drafts from the updated table.
-        if (warp == 0) update_seq<FETCH>(t, b, tokens, row_stride, upd_n_old[b], L, lane, status, counters);
+        if (warp == 0) update_seq<FETCH>(t, b, tokens, row_stride, upd_n_old, L, lane, status, counters);
         __threadfence_block();
         __syncthreads();
     }
@@ -708,6 +708,62 @@ __global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, 
     }
 }
 
+template <int FETCH>
+__global__ void __launch_bounds__(256) cb_draft_kernel(CbTables t, CbTables tf, int T, int crt, int max_depth, int NL, int KF,
+                                                       const int32_t* __restrict__ tokens, int64_t row_stride,
+                                                       const int32_t* __restrict__ seq_len, const int32_t* __restrict__ upd_n_old,
+                                                       int32_t* __restrict__ o_tok, int32_t* __restrict__ o_par,
+                                                       int32_t* __restrict__ o_dep, uint32_t* __restrict__ o_mask,
+                                                       int32_t* __restrict__ o_n, uint32_t* status,
+                                                       unsigned long long* counters) {
+    CB_PDL_ENTRY();
+    extern __shared__ int32_t smem[];
+    const int b = blockIdx.x;
+    draft_body<FETCH>(t, tf, T, crt, max_depth, NL, KF, tokens, row_stride, b, seq_len[b], upd_n_old ? upd_n_old[b] : -1, o_tok, o_par, o_dep,
+                      o_mask, o_n, status, counters, smem);
+}
+
+// Acceptance of one step and update + draft of the next in one launch (the three are a chain per sequence: Fig. 2).  The
+// grid is the acceptance kernel's; the CTA that ends a sequence's acceptance appends the emitted tokens (accepted ones and
+// the bonus token) to the sequence's history, advances its length, and goes on as that sequence's update-and-draft CTA.
+struct AcceptArgs {
+    int V, Dmax, chunk, chunks_per_row;
+    const void* logits; int64_t logits_row_stride;
+    const int32_t* tok; const int32_t* par; const int32_t* dep; const int32_t* n_nodes;
+    unsigned long long* rowmax; uint32_t* ticket;
+    int32_t* n_accept; int32_t* accept_nodes; int32_t* out_tokens; int32_t* target_out;
+};
+
+template <int FETCH, bool BF16>
+__global__ void __launch_bounds__(256) cb_accept_draft_kernel(AcceptArgs a, CbTables t, CbTables tf, int T, int crt, int max_depth, int NL, int KF,
+                                                              int32_t* tokens, int64_t row_stride, int32_t* seq_len,
+                                                              int32_t* o_tok, int32_t* o_par, int32_t* o_dep, uint32_t* o_mask, int32_t* o_n,
+                                                              uint32_t* status, unsigned long long* counters) {
+    CB_PDL_ENTRY();
+    extern __shared__ int32_t smem[];
+    if (!accept_rows<BF16>(T, a.V, a.Dmax, a.chunk, a.chunks_per_row, a.logits, a.logits_row_stride, a.tok, a.par, a.dep, a.n_nodes, a.rowmax,
+                           a.ticket, a.n_accept, a.accept_nodes, a.out_tokens, a.target_out))
+        return;
+    __threadfence_block();
+    __syncthreads();                                            // the walk (first warp) has written the sequence's result
+    const int b = blockIdx.z, tid = threadIdx.x;
+    const int m = __ldcg(&a.n_accept[b]);
+    const int have = min(max(__ldcg(&a.n_nodes[b]), 0), T) > 0 ? m + 1 : 0;   // tokens emitted (an empty tree emits none)
+    const int L = seq_len[b];
+    int L1 = L + have;
+    if (L1 > row_stride) {
+        // no room in the history: nothing is appended and the step is reported; the draft below continues from what is there
+        if (tid == 0) atomicCAS(status, 0u, (uint32_t)CB_ERR_INVALID_ARG);
+        L1 = L;
+    } else if (tid < have) {
+        tokens[(size_t)b * row_stride + L + tid] = __ldcg(&a.out_tokens[(size_t)b * (a.Dmax + 1) + tid]);
+    }
+    __threadfence_block();
+    __syncthreads();
+    if (tid == 0) seq_len[b] = L1;
+    draft_body<FETCH>(t, tf, T, crt, max_depth, NL, KF, tokens, row_stride, b, L1, L, o_tok, o_par, o_dep, o_mask, o_n, status, counters, smem);
+}
+
 }  // namespace
 
 extern "C" cb_status cb_update(cb_ctx* ctx, const int32_t* tokens, int64_t row_stride, const int32_t* n_old,
@@ -833,4 +889,56 @@ extern "C" cb_status cb_update_draft_tree(cb_ctx* ctx, const int32_t* tokens, in
                                           int32_t* tree_depth, uint32_t* tree_mask, int32_t* n_nodes, void* stream) {
     CB_CHECK_ARG(n_old != nullptr);
     return draft_launch(ctx, tokens, row_stride, n_new, n_old, tree_tokens, tree_parent, tree_depth, tree_mask, n_nodes, stream);
+}
+
+extern "C" cb_status cb_accept_update_draft_tree(cb_ctx* ctx, const cb_accept_draft_args* a, void* stream) {
+    CB_CHECK_ARG(ctx && a);
+    CB_CHECK_ARG(a->logits && a->tree_tokens && a->tree_parent && a->tree_depth && a->n_nodes && a->n_accept && a->accept_nodes && a->out_tokens);
+    CB_CHECK_ARG(a->tokens && a->seq_len && a->row_stride >= 1);
+    CB_CHECK_ARG(a->next_tokens && a->next_parent && a->next_depth && a->next_mask && a->next_n_nodes);
+    const cb_config& c = ctx->cfg;
+    CB_CHECK_ARG(a->logits_dtype == CB_DTYPE_F32 || a->logits_dtype == CB_DTYPE_BF16);
+    CB_CHECK_ARG(a->logits_row_stride >= c.vocab);
+    const int esz = a->logits_dtype == CB_DTYPE_F32 ? 4 : 2;
+    CB_CHECK_ARG(((uintptr_t)a->logits & (esz - 1)) == 0);
+    if (c.batch > 65535) return CB_ERR_UNSUPPORTED;
+    const int T = c.max_nodes;
+    // the acceptance grid: about 32 KB of a logits row per CTA, fewer chunks when the batch alone fills the machine
+    int chunk = 32768 / esz;
+    if ((long)c.batch * T >= 8L * ctx->num_sms) chunk *= 4;
+    int cpr = (c.vocab + chunk - 1) / chunk;
+    chunk = ((c.vocab + cpr - 1) / cpr + 7) & ~7;
+    cpr = (c.vocab + chunk - 1) / chunk;
+    AcceptArgs aa;
+    aa.V = c.vocab; aa.Dmax = c.max_depth; aa.chunk = chunk; aa.chunks_per_row = cpr;
+    aa.logits = a->logits; aa.logits_row_stride = a->logits_row_stride;
+    aa.tok = a->tree_tokens; aa.par = a->tree_parent; aa.dep = a->tree_depth; aa.n_nodes = a->n_nodes;
+    aa.rowmax = ctx->d_rowmax; aa.ticket = ctx->d_ticket;
+    aa.n_accept = a->n_accept; aa.accept_nodes = a->accept_nodes; aa.out_tokens = a->out_tokens; aa.target_out = a->target_ids_out;
+    // the drafting CTA's shared memory, as in cb_draft_tree
+    const int NL = min(T, (T - 1) / c.FL + 1);
+    const int FCmax = ctx->has_frozen ? max(c.FC, ctx->frozen.FC) : c.FC;
+    const int KF = max(1, min(FCmax, T - 1));
+    const size_t smem = sizeof(int32_t) * ((size_t)3 * T + (size_t)11 * NL + (size_t)NL * c.FL * KF);
+    if (smem > 200 * 1024) return CB_ERR_UNSUPPORTED;
+    const bool bf = a->logits_dtype == CB_DTYPE_BF16;
+    auto kernel = FCmax <= 32 ? (bf ? cb_accept_draft_kernel<1, true> : cb_accept_draft_kernel<1, false>)
+                              : (bf ? cb_accept_draft_kernel<2, true> : cb_accept_draft_kernel<2, false>);
+    if (smem > 48 * 1024) {
+        static std::mutex mu;
+        static size_t opted[64][4] = {};                       // largest size opted into so far, per device and kernel
+        std::lock_guard<std::mutex> lock(mu);
+        const int d = ctx->device & 63, k = (FCmax <= 32 ? 0 : 2) + (bf ? 1 : 0);
+        if (opted[d][k] < smem) {
+            CB_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            opted[d][k] = smem;
+        }
+    }
+    CbTables tf = {};
+    if (ctx->has_frozen) tf = ctx->frozen;
+    CB_CUDA(cb_launch_pdl(kernel, dim3(cpr, T, c.batch), dim3(256), smem, (cudaStream_t)stream, aa, ctx->tables, tf, T, c.crt, c.max_depth, NL, KF,
+                          a->tokens, a->row_stride, a->seq_len, a->next_tokens, a->next_parent, a->next_depth, a->next_mask, a->next_n_nodes,
+                          ctx->d_status, ctx->d_counters));
+    cb_count_launch(1);
+    return CB_OK;
 }
