@@ -296,7 +296,7 @@ def closed_loop(args, cfg, ctx, toks, lens, tensors, device, frozen):
     from workloads import device as wdev
     from workloads.tensors import TID
     from paper_2511_21699_b200 import Cacheback
-    q, kt, vt, toks_d, out = tensors
+    q, kt, vt, toks_d, out, logits = tensors
     B, T, Dm = cfg.batch, cfg.max_nodes, cfg.max_depth
     KC = 32
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(device)
@@ -334,6 +334,58 @@ def closed_loop(args, cfg, ctx, toks, lens, tensors, device, frozen):
         pos_old.copy_(pos)
         pos.add_(res["n_accept"]).add_(1)
 
+    # The same loop with the target's choice handed over as logits (its arg-max planted in the rows, the stand-in for an LM
+    # head): once with the calls of the loop above, once with cb_accept_update_draft_tree, which takes acceptance, the
+    # append to the history, the update and the next draft in one launch.  Both read the logits; only the launches differ.
+    saved = torch.empty(B, T, dtype=torch.float32, device=device)
+    seq_len = torch.empty(B, **i32)
+
+    def reset_logits_loop():
+        reset()
+        seq_len.copy_(pre_d)
+        cb.cb_draft_tree(toks_d, seq_len, tree)
+
+    def step_logits(fused):
+        cb.cb_tree_attn(q, kp, vp, bt_d, ctx_d, kt, vt, tree["mask"], tree["n_nodes"], out=out, max_ctx=max_ctx)
+        wdev.stream_targets(toks_d, seq_len, tree, cfg.vocab, tgt)
+        wdev.plant_logits(logits, tgt, tree["n_nodes"], saved)
+        if fused:
+            log_n_one.copy_(tree["n_nodes"])                 # the verified tree's sizes are overwritten by the next draft
+            cb.cb_accept_update_draft_tree(tree, logits, toks_d, seq_len, res=res)
+            wdev.plant_logits(logits, tgt, log_n_one, saved, restore=True)
+        else:
+            cb.cb_accept(tree, logits=logits, res=res)
+            wdev.plant_logits(logits, tgt, tree["n_nodes"], saved, restore=True)
+        cb.cb_kv_commit(kp, vp, bt_d, ctx_d, kt, vt, res["n_accept"], res["accept_nodes"])
+        log_emit.add_(res["n_accept"]).add_(1)
+        if not fused:
+            pos_old.copy_(seq_len)
+            seq_len.add_(res["n_accept"]).add_(1)
+            cb.cb_update_draft_tree(toks_d, pos_old, seq_len, tree)
+
+    log_n_one, log_emit = torch.empty(B, **i32), torch.zeros(B, **i32)
+
+    def time_logits_loop(fused):
+        reset_logits_loop()
+        step_logits(fused)
+        stream.synchronize()
+        gl = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gl, stream=stream):
+            for s in range(KC):
+                step_logits(fused)
+        reset_logits_loop()
+        gl.replay()
+        reset_logits_loop()
+        log_emit.zero_()
+        stream.synchronize()
+        e0.record(stream)
+        gl.replay()
+        e1.record(stream)
+        stream.synchronize()
+        emitted = log_emit.cpu().numpy().astype(np.int64)
+        ok = bool(np.array_equal(seq_len.cpu().numpy().astype(np.int64), prefill.astype(np.int64) + emitted))
+        return e0.elapsed_time(e1) / KC, float(emitted.sum()) / (KC * B), ok
+
     stream = torch.cuda.Stream(device=device)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with torch.cuda.stream(stream):
@@ -358,6 +410,8 @@ def closed_loop(args, cfg, ctx, toks, lens, tensors, device, frozen):
             stream.synchronize()
             ms += e0.elapsed_time(e1)
             accs.append(log_acc.cpu().numpy()); toks_out.append(log_tok.cpu().numpy()); nns.append(log_n.cpu().numpy())
+        ms_sep, mat_sep, ok_sep = time_logits_loop(False)
+        ms_fused, mat_fused, ok_fused = time_logits_loop(True)
     st, _ = cb.cb_poll_status()
     assert st == 0, "device status %d in the closed loop" % st
     acc, tok, nn = np.concatenate(accs), np.concatenate(toks_out), np.concatenate(nns)
@@ -374,7 +428,11 @@ def closed_loop(args, cfg, ctx, toks, lens, tensors, device, frozen):
             "emitted_tokens_per_s": steps_tokens / (ms * 1e-3),
             "calls": "cb_update_draft_tree, cb_tree_attn, stream targets (workloads), cb_accept (ids), cb_kv_commit; positions advance on the device",
             "paper_mat_context": {"no_frozen": 1.96, "dual": 2.42, "source": "Table 1, Vicuna 7B on SpecBench, 1x RTX 4090 (context only: other model, other data)"},
-            "frozen_table": frozen is not None}
+            "frozen_table": frozen is not None,
+            "with_logits": {"steps": KC, "ms_per_step_separate_calls": ms_sep, "ms_per_step_fused_call": ms_fused, "mat_separate": mat_sep,
+                            "mat_fused": mat_fused, "lengths_consistent": ok_sep and ok_fused,
+                            "separate_calls": "cb_tree_attn, stream targets + planting (workloads), cb_accept (logits), cb_kv_commit, cb_update_draft_tree",
+                            "fused_call": "cb_tree_attn, stream targets + planting (workloads), cb_accept_update_draft_tree, cb_kv_commit"}}
 
 
 def measure(args, cfg_name, rank, world, device, headline):
@@ -615,9 +673,10 @@ def measure(args, cfg_name, rank, world, device, headline):
     def run_closed_loop():
         if args.no_closed_loop or world > 1:
             return
-        kps.clear(); vps.clear(); lgs.clear()              # the loop brings its own pool (with room to grow)
+        lg0 = lgs[0]
+        kps.clear(); vps.clear(); lgs.clear()              # the loop brings its own pool (with room to grow) and keeps one copy of the logits
         torch.cuda.empty_cache()
-        rec["closed_loop"] = closed_loop(args, cfg, ctx, toks, lens, (q, kt, vt, toks_d, out), device, ft)
+        rec["closed_loop"] = closed_loop(args, cfg, ctx, toks, lens, (q, kt, vt, toks_d, out, lg0), device, ft)
 
     if not headline:
         st, counters = cb.cb_poll_status()

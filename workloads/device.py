@@ -32,6 +32,9 @@ def _load():
         _lib.wl_stream_targets.argtypes = [C.c_void_p, C.c_longlong, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                            C.c_int32, C.c_void_p, C.c_void_p]
         _lib.wl_stream_targets.restype = C.c_int
+        _lib.wl_plant_logits.argtypes = [C.c_void_p, C.c_longlong, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p,
+                                         C.c_int, C.c_void_p]
+        _lib.wl_plant_logits.restype = C.c_int
     return _lib
 
 
@@ -60,3 +63,14 @@ def stream_targets(tokens: torch.Tensor, seq_len: torch.Tensor, tree: dict, junk
     if rc != 0:
         raise RuntimeError("wl_stream_targets failed with CUDA error %d" % rc)
     return out
+
+
+def plant_logits(logits: torch.Tensor, target: torch.Tensor, n_nodes: torch.Tensor, saved: torch.Tensor, restore: bool = False, value: float = 32.0):
+    """Closed-loop stand-in for an LM head (input generation): fp32 logits [B, T, V] get `value` at column target[b, i] of every
+    valid row whose target is a vocabulary id, the entries they replace are kept in saved [B, T]; restore=True puts them back."""
+    B, T, V = logits.shape
+    assert logits.dtype == torch.float32 and logits.stride(2) == 1 and logits.stride(0) == T * logits.stride(1)
+    rc = _load().wl_plant_logits(logits.data_ptr(), logits.stride(1), target.data_ptr(), n_nodes.data_ptr(), B, T, V, float(value),
+                                 saved.data_ptr(), 1 if restore else 0, torch.cuda.current_stream().cuda_stream)
+    if rc != 0:
+        raise RuntimeError("wl_plant_logits failed with CUDA error %d" % rc)

@@ -63,3 +63,23 @@ extern "C" int wl_stream_targets(const int32_t* tokens, long long row_stride, co
     wl_stream_targets_kernel<<<B, T, 0, (cudaStream_t)stream>>>(tokens, row_stride, seq_len, tree_tok, tree_par, tree_dep, n_nodes, B, T, junk_base, target);
     return (int)cudaGetLastError();
 }
+
+// Turns target ids into logits (and back): row (b, i) of the fp32 logits gets `value` at column target[b, i] where that is a
+// vocabulary id, the old entry goes to saved[b, i]; restore != 0 writes the saved entries back.  Input generation only: the
+// closed loop's stand-in for an LM head whose arg-max is the given target.
+__global__ void wl_plant_logits_kernel(float* logits, long long row_stride, const int32_t* target, const int32_t* n_nodes, int B, int T, int V,
+                                       float value, float* saved, int restore) {
+    const int b = blockIdx.x, i = threadIdx.x;
+    if (b >= B || i >= T || i >= n_nodes[b]) return;
+    const int32_t t = target[(long long)b * T + i];
+    if (t < 0 || t >= V) return;
+    float* p = logits + ((long long)b * T + i) * row_stride + t;
+    if (restore) { *p = saved[(long long)b * T + i]; }
+    else { saved[(long long)b * T + i] = *p; *p = value; }
+}
+extern "C" int wl_plant_logits(float* logits, long long row_stride, const int32_t* target, const int32_t* n_nodes, int B, int T, int V, float value,
+                               float* saved, int restore, void* stream) {
+    if (B <= 0 || T <= 0 || T > 1024) return 1;
+    wl_plant_logits_kernel<<<B, T, 0, (cudaStream_t)stream>>>(logits, row_stride, target, n_nodes, B, T, V, value, saved, restore);
+    return (int)cudaGetLastError();
+}
