@@ -10,13 +10,15 @@
 // So the run is reduced first, with one thread per window and no warp owning a leader's history:
 //   1. every window finds or claims the slot of its (leader, follower) pair in a scratch hash table and of its leader in a
 //      second one, and raises their "last index" with atomicMax; the thread that creates a pair counts it for its leader;
-//   2. every leader takes a range of the group array (atomicAdd on a cursor), 3. every pair writes itself into its
-//      leader's range;
-//   4. one warp per leader finds or creates the table entry, sets the leader's stamp, and inserts the leader's pairs with
-//      the usual follower-list code, or only the FC latest of them when there are more (threshold by bisection on the last
-//      index).  Those FC are newer than anything stored, so inserting them in any order evicts stored followers oldest
-//      first and never one of them: the result is the sequential one.  Which place a follower takes in the entry, and
-//      which entry id a leader gets, may differ from the sequential run; nothing reads either.
+//   2. every leader takes a range of the group array (a block scan over 256 slots, then one atomicAdd on a cursor),
+//   3. every pair writes itself into its leader's range;
+//   4. the leaders are applied to the table, 32 slots per warp: a leader that is not in the table yet and has few followers
+//      is written by one lane alone (entry id from the leader count, key, followers, stamps), every other one by the whole
+//      warp, which finds or creates the entry, sets the leader's stamp, and inserts the leader's pairs with the usual
+//      follower-list code, or only the FC latest of them when there are more (threshold by bisection on the last index).
+//      Those FC are newer than anything stored, so inserting them in any order evicts stored followers oldest first and
+//      never one of them: the result is the sequential one.  Which place a follower takes in the entry, and which entry id
+//      a leader gets, may differ from the sequential run; nothing reads either.
 // Keys are compared by reading the tokens at the position a slot's first claimant recorded.  All loops are bounded.
 #pragma once
 
