@@ -73,15 +73,21 @@ __device__ __forceinline__ int cb_max_row_groups(const CbAttnParams& p) { return
 
 // Warp-collective: total weight of all sequences, and the (row group, sequence) holding global position g (with the
 // global index at which that sequence's units of that row group start).  Every lane gets the results.
-__device__ __forceinline__ long long cb_sched_total(const CbAttnParams& p, int lane) {
+// max_row_tiles (optional): the largest number of row tiles that any sequence's tree has.
+__device__ __forceinline__ long long cb_sched_total(const CbAttnParams& p, int lane, int* max_row_tiles = nullptr) {
     long long tot = 0;
+    int mt = 0;
     for (int base = 0; base < p.B; base += 32) {
         const int b = base + lane;
-        long long w = b < p.B ? cb_seq_shape(p, b).W : 0;
+        CbSeqShape s = {};
+        if (b < p.B) s = cb_seq_shape(p, b);
+        long long w = b < p.B ? s.W : 0;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) w += __shfl_xor_sync(CB_FULL, w, o);
         tot += w;
+        mt = max(mt, b < p.B ? s.mtn : 0);
     }
+    if (max_row_tiles) *max_row_tiles = __reduce_max_sync(CB_FULL, mt);
     return tot;
 }
 __device__ __forceinline__ void cb_sched_locate(const CbAttnParams& p, long long g, int lane, int* rg_out, int* b_out, long long* pre_out) {

@@ -10,7 +10,8 @@
 //                 by the ring
 //   warp 1        MMA issuer (one lane): S = Q K^T into TMEM, then O += P V with P read from TMEM;
 //                 owns the TMEM allocation (S0, S1, O0, O1: 4 x 128 columns)
-//   warp 2        TMA loader for the query tiles of each unit
+//   warp 2        TMA loader for the query tiles of each unit; in launches where every unit has one row tile it also issues
+//                 S = Q K^T, and warp 1 only O += P V (two issuing threads, see two_issuers below)
 //   warp 3        writes the zero rows of padding nodes (node >= n_nodes), then TMA producer for the V tiles
 //   warps 4..7    softmax warpgroup 0, warps 8..11 softmax warpgroup 1: one thread per query row; S from
 //                 TMEM to registers, fp32 online softmax in the log2 domain with lazy rescaling of O,
@@ -42,7 +43,7 @@ struct Cfg {
     static constexpr uint32_t OFF_RING = 2 * Q_BYTES;
     static constexpr uint32_t OFF_BAR = OFF_RING + NSLOT * TILE_BYTES;
     // slot_full[NSLOT], slot_free[NSLOT], q_full, q_free, s_full0, p_ready[2], o_free[2], cluster_ready, cluster_data
-    static constexpr int NBAR = 2 * NSLOT + 2 + 7;
+    static constexpr int NBAR = 2 * NSLOT + 2 + 7 + 2;       // ... and pv_done[2]
     static constexpr uint32_t OFF_MISC = OFF_BAR + NBAR * 8;  // schedule, tmem base, abort flag
     static constexpr uint32_t SMEM = OFF_MISC + 96;
     static constexpr uint32_t SMEM_ALLOC = SMEM + 1024;      // slack to align the base to 1024 bytes
@@ -68,6 +69,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     const uint32_t bar0 = sbase + C::OFF_BAR;
     auto bar_full = [&](int s) { return bar0 + 8u * s; };
     auto bar_free = [&](int s) { return bar0 + 8u * (C::NSLOT + s); };
+    auto slot_base = [&](uint32_t s) { return sbase + C::OFF_RING + s * C::TILE_BYTES; };
     const uint32_t bar_qfull = bar0 + 8u * (2 * C::NSLOT), bar_qfree = bar_qfull + 8u;
     // Completion of the tensor core's work is signalled with as few commits as possible (a second commit behind the
     // same MMA block stalls the issuer): a ring slot's "free" barrier doubles as "the S product that read this K tile is
@@ -78,9 +80,11 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     auto bar_pready = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 3 + s); };
     auto bar_ofree = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 5 + s); };
     const uint32_t bar_cready = bar0 + 8u * (2 * C::NSLOT + 7), bar_cdata = bar_cready + 8u;   // cluster mode only
+    auto bar_pvdone = [&](int s) { return bar0 + 8u * (2 * C::NSLOT + 9 + s); };               // two issuing threads only (see below)
     SchedSmem* s_sched = reinterpret_cast<SchedSmem*>(sgen + C::OFF_MISC);
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(sgen + C::OFF_MISC + 64);
     volatile int* s_abort = reinterpret_cast<volatile int*>(sgen + C::OFF_MISC + 68);
+    volatile int* s_one_row = reinterpret_cast<volatile int*>(sgen + C::OFF_MISC + 72);   // every unit of the launch has one row tile
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
@@ -100,6 +104,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                 mbar_init(bar_pready(s), 256); mbar_init(bar_ofree(s), 128);
             }
             mbar_init(bar_cready, p.cs > 0 ? (uint32_t)p.cs : 1u); mbar_init(bar_cdata, 128);
+            mbar_init(bar_pvdone(0), 1); mbar_init(bar_pvdone(1), 1);
             *s_abort = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             tma_prefetch_desc(&maps.k_pool); tma_prefetch_desc(&maps.v_pool); tma_prefetch_desc(&maps.q);
@@ -119,15 +124,20 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             s_sched->c_t0 = sh.RG > 0 ? (int)((long long)sh.tiles * rank / p.cs) : 0;
             s_sched->c_t1 = sh.RG > 0 ? (int)((long long)sh.tiles * (rank + 1) / p.cs) : 0;
             s_sched->g0 = 0; s_sched->g1 = 0; s_sched->pre0 = 0; s_sched->b0 = 0; s_sched->rg0 = 0;
+            *s_one_row = 1;
         }
     } else if (warp == 0) {
         // this CTA's range of the global tile sequence
-        const long long tot = cb_sched_total(p, lane);
+        int max_rt = 0;
+        const long long tot = cb_sched_total(p, lane, &max_rt);
         const long long g0 = cb_range_start(tot, p.nc, cta), g1 = cb_range_start(tot, p.nc, cta + 1);
         int b0 = 0, rg0 = 0;
         long long pre0 = 0;
         if (g0 < g1) cb_sched_locate(p, g0, lane, &rg0, &b0, &pre0);
-        if (lane == 0) { s_sched->g0 = g0; s_sched->g1 = g1; s_sched->b0 = b0; s_sched->rg0 = rg0; s_sched->pre0 = pre0; }
+        if (lane == 0) {
+            s_sched->g0 = g0; s_sched->g1 = g1; s_sched->b0 = b0; s_sched->rg0 = rg0; s_sched->pre0 = pre0;
+            *s_one_row = (p.MT == 1 || max_rt <= 1) ? 1 : 0;
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -135,6 +145,13 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
     const uint32_t tmem = *s_tmem;
     const long long g0 = s_sched->g0, g1 = s_sched->g1, pre0 = s_sched->pre0;
     const int b0 = s_sched->b0, rg0 = s_sched->rg0;
+    // When no unit of the launch has two row tiles (the same for every CTA: it follows from n_nodes alone), the products of a
+    // key tile get an issuing thread each: warp 2's thread, which loads the query tile, issues S = Q K^T, warp 1's thread
+    // issues O += P V.  One thread issuing both spends about 2.0 k cycles per key tile in the two blocks and its loop, and the
+    // next S follows the P.V it has to wait for; with two threads the next S only waits for the completion of the P.V that
+    // read its buffer two tiles before, and the softmax warpgroup (1.9 k cycles per tile) is what a tile costs.
+    const bool two_issuers = *s_one_row != 0;
+    constexpr uint32_t ns = (uint32_t)C::NSLOT;
     CbWalker wk;
     if (p.cs > 0) {
         // the peers' barriers must exist before anything arrives on them
@@ -192,12 +209,12 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     int page = page_next;
                     if (i + 1 < u.t1) page_next = page_of(i + 1);
                     if (!cb_dbg_in(page, p.num_pages + 1, p.status)) page = p.num_pages;   // the copy then fills zeros
-                    const uint32_t sl = seq % C::NSLOT;
-                    if (seq >= (uint32_t)C::NSLOT && !(ok = mbar_wait(bar_free(sl), (seq / C::NSLOT - 1) & 1, s_abort, p.status))) break;
+                    const uint32_t sl = seq % ns;
+                    if (seq >= ns && !(ok = mbar_wait(bar_free(sl), (seq / ns - 1) & 1, s_abort, p.status))) break;
                     if (lane == 0) mbar_expect_tx(bar_full(sl), C::TILE_BYTES);
                     __syncwarp();
                     if (active) {
-                        const uint32_t dst = sbase + C::OFF_RING + sl * C::TILE_BYTES + dblk * (CB_KT * 128) + j * 2048;
+                        const uint32_t dst = slot_base(sl) + dblk * (CB_KT * 128) + j * 2048;
                         if (i < nct) tma_load_4d_hint(dst, isV ? &maps.v_pool : &maps.k_pool, bar_full(sl), dblk * 64, u.kh, 0, page, pol);
                         else tma_load_4d(dst, isV ? &maps.v_tree : &maps.k_tree, bar_full(sl), dblk * 64, u.kh, 16 * j, u.b);
                     }
@@ -219,8 +236,32 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                 auto issue_pv = [&](int ol, int buf, uint32_t vslot, bool accum) {
                     mma_pv_block(tmem + C::O_COL + ol * D, tmem + buf * 128, v_lo0 + vslot * (C::TILE_BYTES >> 4), idesc_o, accum ? 1u : 0u);
                 };
+                if (two_issuers) {
+                    // O += P V only (S is issued by warp 2's thread).  After every product one more commit reports it on the
+                    // barrier of the S buffer whose P it read: the next S into that buffer waits for it.
+                    uint32_t c_of0 = 0;
+                    while (ok && wk.next(p, &u)) {
+                        const uint32_t seq0 = seq;
+                        for (int i = u.t0; ok && i < u.t1; ++i) {
+                            const int buf = (i - u.t0) & 1;
+                            const uint32_t vseq = seq0 + 2u * (uint32_t)(i - u.t0) + 1u, vs = vseq % ns;
+                            if (!(ok = mbar_wait(bar_full(vs), (vseq / ns) & 1, s_abort, p.status))) break;
+                            if (!(ok = mbar_wait(bar_pready(buf), c_p[buf] & 1, s_abort, p.status))) break;
+                            ++c_p[buf];
+                            if (i == u.t0) {
+                                if (c_of0 > 0 && !(ok = mbar_wait(bar_ofree(0), (c_of0 - 1) & 1, s_abort, p.status))) break;
+                                ++c_of0;
+                            }
+                            tc_fence_after();
+                            mma_pv_block(tmem + C::O_COL, tmem + buf * 128, desc_lo(slot_base(vs), CB_KT * 128), idesc_o, i > u.t0 ? 1u : 0u);
+                            tc_commit(bar_free(vs));
+                            tc_commit(bar_pvdone(buf));
+                        }
+                        seq = seq0 + 2u * (uint32_t)(u.t1 - u.t0);
+                    }
+                }
                 CbUnit un;
-                    bool have = wk.next(p, &un);
+                    bool have = !two_issuers && wk.next(p, &un);
                 while (ok && have) {
                     u = un;
                     const bool two = u.nrt == 2;
@@ -294,7 +335,36 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             // ------------------------------------------------------------------ query loader
             if (lane == 0) {
                 uint32_t uq = 0;
-                while (wk.next(p, &u)) {
+                if (two_issuers) {
+                    // query tile, then S = Q K^T of every key tile of the unit.  The k-th S into a buffer waits for the
+                    // completion of the P.V that read the (k-1)-th P from it.
+                    constexpr uint32_t idesc_s = make_idesc(128, CB_KT, false);
+                    const uint32_t q_lo0 = desc_lo(sbase + C::OFF_Q, 16);
+                    uint32_t seq = 0, c_s[2] = {0u, 0u};
+                    bool ok = true;
+                    while (ok && wk.next(p, &u)) {
+                        if (uq > 0 && !(ok = mbar_wait(bar_qfree, (uq - 1) & 1, s_abort, p.status))) break;
+                        mbar_expect_tx(bar_qfull, (uint32_t)(C::DB * RT * 128));
+                        for (int db = 0; db < C::DB; ++db)
+                            tma_load_4d(sbase + C::OFF_Q + db * (CB_MT * 128), &maps.q, bar_qfull, db * 64, u.kh * p.G, u.rg * 2 * p.NPT, u.b);
+                        if (!(ok = mbar_wait(bar_qfull, uq & 1, s_abort, p.status))) break;
+                        ++uq;
+                        const uint32_t seq0 = seq;
+                        for (int i = u.t0; ok && i < u.t1; ++i) {
+                            const int buf = (i - u.t0) & 1;
+                            const uint32_t kseq = seq0 + 2u * (uint32_t)(i - u.t0), ks = kseq % ns;
+                            if (!(ok = mbar_wait(bar_full(ks), (kseq / ns) & 1, s_abort, p.status))) break;
+                            if (c_s[buf] > 0 && !(ok = mbar_wait(bar_pvdone(buf), (c_s[buf] - 1) & 1, s_abort, p.status))) break;
+                            ++c_s[buf];
+                            tc_fence_after();
+                            mma_s_block<D>(tmem + buf * 128, q_lo0, desc_lo(slot_base(ks), 16), idesc_s);
+                            tc_commit(bar_free(ks));
+                            if (i == u.t1 - 1) tc_commit(bar_qfree);
+                        }
+                        seq = seq0 + 2u * (uint32_t)(u.t1 - u.t0);
+                    }
+                }
+                while (!two_issuers && wk.next(p, &u)) {
                     if (uq > 0 && !mbar_wait(bar_qfree, (uq - 1) & 1, s_abort, p.status)) break;
                     mbar_expect_tx(bar_qfull, (uint32_t)(u.nrt * C::DB * RT * 128));
                     for (int rt = 0; rt < u.nrt; ++rt)
@@ -363,7 +433,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                 // its own, given when it has seen the tile's S, so the products cannot run more than a tile ahead of it.
                 for (int i = u.t0; ok && i < u.t1; ++i) {
                     const uint32_t kseq = seq0 + 2u * (uint32_t)(i - u.t0);
-                    ok = mbar_wait(bar_free(kseq % C::NSLOT), (kseq / C::NSLOT) & 1, s_abort, p.status);
+                    ok = mbar_wait(bar_free(kseq % ns), (kseq / ns) & 1, s_abort, p.status);
                     mbar_arrive(bar_pready((i - u.t0) & 1));
                 }
                 have = fetch_next();
@@ -373,7 +443,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
             // every PV up to tile i is done when tile i's V slot is released.
             auto wait_pv = [&](int i) {
                 const uint32_t vseq = seq0 + 2u * (uint32_t)(i - u.t0) + 1u;
-                return mbar_wait(bar_free(vseq % C::NSLOT), (vseq / C::NSLOT) & 1, s_abort, p.status);
+                return mbar_wait(bar_free(vseq % ns), (vseq / ns) & 1, s_abort, p.status);
             };
             const int rt = u.rg * 2 + wg;
             const int node = rt * p.NPT + row / p.G, g = row % p.G, h = u.kh * p.G + g;
@@ -388,7 +458,7 @@ cb_attn_tc_kernel(const CbAttnParams p, const __grid_constant__ TcMaps maps) {
                     ++c_s0;
                 } else {
                     const uint32_t kseq = seq0 + 2u * (uint32_t)(i - u.t0);
-                    if (!(ok = mbar_wait(bar_free(kseq % C::NSLOT), (kseq / C::NSLOT) & 1, s_abort, p.status))) break;
+                    if (!(ok = mbar_wait(bar_free(kseq % ns), (kseq / ns) & 1, s_abort, p.status))) break;
                 }
                 if (warp_active) {
                     tc_fence_after();
