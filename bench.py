@@ -58,13 +58,13 @@ def parse(argv=None):
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one cb_attn_tc_kernel launch with full trees, from the ncu
 # captures summarised under profiles/.  Reported only while the kernel sources still hash to the captured ones; after any
 # change to them the figure is stale and `traffic` is null until the capture is redone.
-ATTN_TRAFFIC = {"sources_sha1": "326f51a8dad08b723b956b28c58e4dac1519bd3b",
-                "bytes_per_launch": {"c2_7b": 70.1e6, "c3_8b_gqa": 558.4e6, "c4_13b_turns": 2767.2e6},
+ATTN_TRAFFIC = {"sources_sha1": "631ae1a4edeb073d1c842aef25b5ff4467c347b4",
+                "bytes_per_launch": {"c2_7b": 70.2e6, "c3_8b_gqa": 557.6e6, "c4_13b_turns": 2767.4e6},
                 "source": {k: "profiles/cb_attn_tc_kernel_c2_c3_c4_c5b8.md" for k in ("c2_7b", "c3_8b_gqa", "c4_13b_turns")},
                 # config 5 holds 25 GB and runs 20 ms per launch: too large to capture.  The same shape at batch 8 was captured
-                # (1,317.9 + 8.0 and 1,217.3 + 8.9 MB per launch); keys and values are streamed per sequence, so the traffic is taken
+                # (1,405.0 + 8.4 and 1,432.1 + 8.4 MB per launch); keys and values are streamed per sequence, so the traffic is taken
                 # to grow with the batch: mean x 128 / 8.
-                "scaled": {"c5_70b_long": (1276.1e6 * 16.0,
+                "scaled": {"c5_70b_long": (1427.0e6 * 16.0,
                                            "profiles/cb_attn_tc_kernel_c2_c3_c4_c5b8.md: c5_70b_b8 (same shape, batch 8), mean of two captures "
                                            "x 16 sequences' worth; not a capture of this workload")}}
 ATTN_SOURCES = ("cb_attn_tc.cu", "cb_tc_dev.cuh", "cb_attn_pair.cuh", "cb_attn.cuh", "cb_attn.cu")
